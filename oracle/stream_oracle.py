@@ -1,0 +1,180 @@
+"""ctypes loader for the plain-C oracle in ``stream_oracle.c``.
+
+Test infrastructure only. It is compiled with gcc on the machine that uses it (the object is
+keyed by the source text, the flags and the CPU model, so a copy built elsewhere is never
+reused) and holds no arithmetic of its own: every number comes from the C file.
+
+Arrays are numpy, contiguous: Q ``[batch, n_q_heads, T, d]``, K/V ``[batch, n_kv_heads, T, d]``,
+dtype float32, or uint16 holding bf16 bit patterns.
+"""
+from __future__ import annotations
+
+import ctypes
+import hashlib
+import os
+import platform
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "stream_oracle.c")
+_FLAGS = ["-O3", "-march=native", "-ffp-contract=off", "-fopenmp", "-fPIC", "-shared", "-std=c11"]
+
+SCORE_CACHE = 1  # so_build_mask_rows flag: reuse s(q, r) within a row (same values, fewer tiles)
+
+
+class _CProblem(ctypes.Structure):
+    _fields_ = [
+        ("batch", ctypes.c_int32), ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
+        ("T", ctypes.c_int64),
+        ("d", ctypes.c_int32), ("block_q", ctypes.c_int32), ("block_k", ctypes.c_int32),
+        ("k_top", ctypes.c_int32), ("causal", ctypes.c_int32), ("dtype", ctypes.c_int32),
+    ]
+
+
+@dataclass(frozen=True)
+class OracleProblem:
+    batch: int
+    n_q_heads: int
+    n_kv_heads: int
+    T: int
+    d: int
+    block_q: int
+    block_k: int
+    k_top: int
+    causal: bool = True
+    dtype: str = "f32"  # "f32" or "bf16"
+
+    def c(self) -> _CProblem:
+        return _CProblem(self.batch, self.n_q_heads, self.n_kv_heads, self.T, self.d, self.block_q,
+                         self.block_k, self.k_top, int(self.causal), {"f32": 0, "bf16": 1}[self.dtype])
+
+
+def _cpu_tag() -> str:
+    model = platform.processor()
+    try:
+        with open("/proc/cpuinfo") as fh:
+            for line in fh:
+                if line.startswith(("model name", "flags")):
+                    model += line
+                    if line.startswith("flags"):
+                        break
+    except OSError:
+        pass
+    return model
+
+
+def _lib_path() -> str:
+    with open(_SRC, "rb") as fh:
+        key = hashlib.sha256(fh.read() + " ".join(_FLAGS).encode() + _cpu_tag().encode()).hexdigest()[:16]
+    return os.path.join(_HERE, "_build", f"libstream_oracle_{key}.so")
+
+
+def build() -> str:
+    """Compile the oracle for this machine if that has not been done; return the library path."""
+    path = _lib_path()
+    if not os.path.exists(path):
+        os.makedirs(os.path.dirname(path), exist_ok=True)
+        tmp = f"{path}.{os.getpid()}.tmp"
+        subprocess.run(["gcc", *_FLAGS, _SRC, "-o", tmp, "-lm"], check=True)
+        os.replace(tmp, path)
+    return path
+
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        vp, i64p = ctypes.c_void_p, ctypes.c_void_p
+        lib.so_num_query_blocks.restype = ctypes.c_int64
+        lib.so_num_query_blocks.argtypes = [ctypes.POINTER(_CProblem)]
+        lib.so_num_rows.restype = ctypes.c_int64
+        lib.so_num_rows.argtypes = [ctypes.POINTER(_CProblem)]
+        lib.so_threads.restype = ctypes.c_int
+        lib.so_tile_score.restype = ctypes.c_float
+        lib.so_tile_score.argtypes = [ctypes.POINTER(_CProblem), vp, vp] + [ctypes.c_int64] * 4
+        lib.so_build_mask_rows.restype = ctypes.c_int
+        lib.so_build_mask_rows.argtypes = [ctypes.POINTER(_CProblem), vp, vp, i64p, ctypes.c_int64,
+                                           vp, vp, vp, vp, ctypes.c_int, ctypes.c_int]
+        lib.so_sparse_attention_rows.restype = ctypes.c_int
+        lib.so_sparse_attention_rows.argtypes = [ctypes.POINTER(_CProblem), vp, vp, vp, i64p, ctypes.c_int64,
+                                                 vp, ctypes.c_double, vp]
+        _lib = lib
+    return _lib
+
+
+def _check(p: OracleProblem, x: np.ndarray, heads: int, name: str) -> np.ndarray:
+    want = np.float32 if p.dtype == "f32" else np.uint16
+    if x.dtype != want or not x.flags["C_CONTIGUOUS"] or x.shape != (p.batch, heads, p.T, p.d):
+        raise ValueError(f"{name}: need contiguous {np.dtype(want)} array of shape {(p.batch, heads, p.T, p.d)}")
+    return x
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def threads() -> int:
+    return int(_load().so_threads())
+
+
+def num_query_blocks(p: OracleProblem) -> int:
+    return int(_load().so_num_query_blocks(ctypes.byref(p.c())))
+
+
+def num_rows(p: OracleProblem) -> int:
+    return int(_load().so_num_rows(ctypes.byref(p.c())))
+
+
+def tile_score(p: OracleProblem, q: np.ndarray, k: np.ndarray, b: int, h: int, qb: int, r: int) -> float:
+    _check(p, q, p.n_q_heads, "q"), _check(p, k, p.n_kv_heads, "k")
+    return float(_load().so_tile_score(ctypes.byref(p.c()), _ptr(q), _ptr(k), b, h, qb, r))
+
+
+def build_mask_rows(p: OracleProblem, q: np.ndarray, k: np.ndarray, rows=None, *, n_it: int = -1,
+                    score_cache: bool = False, want_scores: bool = False):
+    """Algorithm 2 for ``rows`` (flat row ids; ``None`` = every row).
+
+    Returns a dict: ``mask`` int32 [n, k_top] (ascending block indices, -1 padded), ``min_gap``
+    float32 [n], ``tiles`` int64 [n] and, if asked, ``scores`` float32 [n, k_top].
+    """
+    _check(p, q, p.n_q_heads, "q"), _check(p, k, p.n_kv_heads, "k")
+    lib = _load()
+    rows_arr = None if rows is None else np.ascontiguousarray(rows, dtype=np.int64)
+    n = num_rows(p) if rows_arr is None else rows_arr.shape[0]
+    mask = np.empty((n, p.k_top), np.int32)
+    gap = np.empty((n,), np.float32)
+    tiles = np.empty((n,), np.int64)
+    scores = np.empty((n, p.k_top), np.float32) if want_scores else None
+    rc = lib.so_build_mask_rows(ctypes.byref(p.c()), _ptr(q), _ptr(k), _ptr(rows_arr), n, _ptr(mask),
+                                _ptr(scores), _ptr(gap), _ptr(tiles), n_it, SCORE_CACHE if score_cache else 0)
+    if rc:
+        raise RuntimeError(f"so_build_mask_rows failed with {rc}")
+    out = {"mask": mask, "min_gap": gap, "tiles": tiles}
+    if want_scores:
+        out["scores"] = scores
+    return out
+
+
+def sparse_attention_rows(p: OracleProblem, q: np.ndarray, k: np.ndarray, v: np.ndarray, mask: np.ndarray,
+                          rows=None, *, scale: float | None = None) -> np.ndarray:
+    """Eq. 2 restricted to the blocks in ``mask`` ([n, k_top]); returns fp64 [n, block_q, d]."""
+    _check(p, q, p.n_q_heads, "q"), _check(p, k, p.n_kv_heads, "k"), _check(p, v, p.n_kv_heads, "v")
+    lib = _load()
+    rows_arr = None if rows is None else np.ascontiguousarray(rows, dtype=np.int64)
+    n = num_rows(p) if rows_arr is None else rows_arr.shape[0]
+    mask = np.ascontiguousarray(mask, dtype=np.int32)
+    if mask.shape != (n, p.k_top):
+        raise ValueError(f"mask: need shape {(n, p.k_top)}, got {mask.shape}")
+    out = np.empty((n, p.block_q, p.d), np.float64)
+    s = float(scale) if scale is not None else 1.0 / float(np.sqrt(p.d))
+    rc = lib.so_sparse_attention_rows(ctypes.byref(p.c()), _ptr(q), _ptr(k), _ptr(v), _ptr(rows_arr), n,
+                                      _ptr(mask), s, _ptr(out))
+    if rc:
+        raise RuntimeError(f"so_sparse_attention_rows failed with {rc}")
+    return out

@@ -1,0 +1,158 @@
+/*
+ * libstream: C ABI of the B200 (sm_100a) implementation of Stream sparse-mask estimation and
+ * the block-sparse attention pass that consumes the mask.
+ *
+ * Conventions for every entry point
+ *   - Plain C types only. Unless a parameter says HOST, every data pointer is a DEVICE pointer
+ *     owned by the caller; the library never allocates or frees device memory and keeps no
+ *     state between calls apart from the thread-local error text.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = default stream)
+ *     and the call returns after enqueue unless stated otherwise.
+ *   - Every failure is a returned status; nothing aborts or throws. Arguments are validated on
+ *     the host before anything is launched. stream_last_error() gives the text of the last
+ *     failure on the calling thread.
+ *   - Tensors: Q is [batch, n_q_heads, T, d], K and V are [batch, n_kv_heads, T, d], addressed
+ *     with the element strides in the problem struct (innermost stride 1). Query head h reads
+ *     kv head h / (n_q_heads / n_kv_heads). dtype is fp32 or bf16 for Q, K, V and the attention
+ *     output alike. Inputs must be finite.
+ *   - A "row" is one (batch, query head, query block); there are ceil(T / block_q) query
+ *     blocks. The mask is int32 [batch, n_q_heads, ceil(T / block_q), k_top], contiguous: per
+ *     row the kept key-block indices (0-based; block r covers tokens r*block_k ..), strictly
+ *     ascending, then -1 padding.
+ */
+#ifndef STREAM_H_
+#define STREAM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    STREAM_OK = 0,
+    STREAM_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, bad stride, bad enum */
+    STREAM_ERR_UNSUPPORTED = 2, /* valid request that no kernel here covers (see stream_problem) */
+    STREAM_ERR_WORKSPACE = 3,   /* workspace or staging buffer missing, misaligned or too small */
+    STREAM_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed; text in stream_last_error */
+    STREAM_ERR_DEVICE_CHECK = 5 /* a kernel gave up on a bounded wait; see stream_read_stats */
+} stream_status;
+
+typedef enum { STREAM_F32 = 0, STREAM_BF16 = 1 } stream_dtype;
+
+typedef enum {
+    STREAM_IMPL_AUTO = 0,    /* tensor-core kernels when the shape allows, else the generic ones */
+    STREAM_IMPL_GENERIC = 1, /* fp32-FMA kernels: any dtype, d in {16,32,64,128}, blocks 1..64 */
+    STREAM_IMPL_TENSOR = 2   /* tcgen05 kernels only: bf16, d = 128, block_q = block_k = 64,
+                                k_top <= 64, causal; otherwise STREAM_ERR_UNSUPPORTED */
+} stream_impl;
+
+typedef struct {
+    int32_t batch;          /* independent problems (e.g. layers); >= 1 */
+    int32_t n_q_heads;      /* >= 1 */
+    int32_t n_kv_heads;     /* >= 1 and divides n_q_heads */
+    int64_t T;              /* tokens, >= 1; need not be a multiple of the block sizes */
+    int32_t d;              /* head dimension */
+    int32_t block_q;        /* b_q */
+    int32_t block_k;        /* b_k */
+    int32_t k_top;          /* k: key blocks kept per query block = row width of the mask; 1..1024 */
+    int32_t causal;         /* 1: C is lower triangular; 0: C is all ones (Algorithm 1) */
+    int32_t dtype;          /* stream_dtype */
+    int32_t impl;           /* stream_impl */
+    int64_t q_stride_b, q_stride_h, q_stride_t;    /* elements */
+    int64_t kv_stride_b, kv_stride_h, kv_stride_t; /* elements; K and V share them */
+} stream_problem;
+
+/* Counters a mask build leaves in the first bytes of its workspace. */
+typedef struct {
+    uint64_t tiles_scored; /* (row, representative key block) tiles whose score was computed */
+    uint64_t rows;         /* rows finished */
+    uint32_t error;        /* 0, or a code saying which bounded wait ran out (kernel returned early) */
+    uint32_t error_info;
+} stream_stats;
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int stream_version(void);
+
+/* Text of the most recent failure on this thread ("" if none). The pointer stays valid until the
+ * thread's next failing call. */
+const char *stream_last_error(void);
+
+/*
+ * Bytes of device workspace stream_build_mask needs for this problem (a small header holding
+ * stream_stats and the work counter of the persistent kernels; O(1), never grows with T).
+ * Returns 0 if the problem is invalid or unsupported.
+ */
+size_t stream_workspace_bytes(const stream_problem *p);
+
+/*
+ * Stream mask estimation (Algorithm 2 of the paper; Algorithm 1 when causal == 0).
+ *
+ * For every row: start from k_top nodes tiling the N_k key blocks, and for ceil(log2 N_k) levels
+ * split every node in two, score each branch by the masked maximum token-level dot product
+ * (Eq. 4) between the query block and the branch's first allowed key block, keep the k_top best
+ * branches (higher fp32 score, then lower block index), and finally emit the first allowed block
+ * of every surviving node. Levels that cannot change the result (all nodes single blocks) are
+ * skipped, and a left branch reuses its parent's score (same tile, same value).
+ *
+ *   q, k       device, dtype of the problem, strided as described above; read only
+ *   mask_out   device int32 [batch, n_q_heads, ceil(T/block_q), k_top]; fully overwritten
+ *   score_out  device float32, same shape, or NULL: block score of every kept block, -inf padded
+ *   workspace  device, 256-byte aligned, >= stream_workspace_bytes(p); overwritten. After the
+ *              stream has drained, stream_read_stats(workspace, ...) returns this call's counters.
+ *
+ * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE before any launch; CUDA if a launch fails.
+ */
+stream_status stream_build_mask(const stream_problem *p, const void *q, const void *k, int32_t *mask_out,
+                                float *score_out, void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Block-sparse attention under a Stream mask (Eq. 2 of the paper; the product QK^T * C * M of
+ * Figure 1): for every query token, softmax(scale * q.k) over the keys of the row's kept blocks
+ * that C allows (element-level causal test inside a block, keys beyond T excluded), times V.
+ * Softmax statistics and the output accumulate in fp32; a token that no kept key is allowed for
+ * gets zeros.
+ *
+ *   q, k, v    device, dtype of the problem; read only
+ *   mask       device int32 [batch, n_q_heads, ceil(T/block_q), k_top] as written by
+ *              stream_build_mask; entries < 0 are skipped; valid entries must be < ceil(T/block_k)
+ *   scale      logit scale; <= 0 selects 1/sqrt(d)
+ *   out        device, dtype of the problem, contiguous [batch, n_q_heads, T, d]; overwritten
+ */
+stream_status stream_sparse_attention(const stream_problem *p, const void *q, const void *k, const void *v,
+                                      const int32_t *mask, float scale, void *out, void *cuda_stream);
+
+/*
+ * Synchronous read-back of the counters left by the last stream_build_mask that used this
+ * workspace. Waits for `cuda_stream` to drain, copies the header to *out (HOST pointer) and
+ * returns STREAM_ERR_DEVICE_CHECK if the kernel recorded a bounded wait that ran out.
+ */
+stream_status stream_read_stats(const void *workspace, stream_stats *out, void *cuda_stream);
+
+/*
+ * Bytes of device staging stream_run_host needs: room for Q, K, V, the mask, the output and the
+ * mask workspace, each 256-byte aligned. 0 if the problem is invalid or unsupported.
+ */
+size_t stream_host_staging_bytes(const stream_problem *p);
+
+/*
+ * The whole path from HOST memory: copy Q, K, V to the device, build the mask, run the sparse
+ * attention, copy mask and output back. Strides in *p describe the HOST tensors, which must be
+ * dense ([batch, heads, T, d] contiguous); pinned host memory makes the copies asynchronous.
+ *
+ *   q_host, k_host, v_host   HOST, read only
+ *   mask_host                HOST int32 [batch, n_q_heads, ceil(T/block_q), k_top]
+ *   out_host                 HOST, dtype of the problem, [batch, n_q_heads, T, d]
+ *   staging                  DEVICE, 256-byte aligned, >= stream_host_staging_bytes(p)
+ * Returns after everything is enqueued on cuda_stream; the host buffers are valid once the
+ * stream has been synchronised.
+ */
+stream_status stream_run_host(const stream_problem *p, const void *q_host, const void *k_host, const void *v_host,
+                              int32_t *mask_host, void *out_host, float scale, void *staging,
+                              size_t staging_bytes, void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* STREAM_H_ */

@@ -1,0 +1,207 @@
+// extern "C" boundary of libstream: argument validation, geometry, dispatch. See stream.h.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+
+#include "common.cuh"
+
+namespace stream {
+
+static thread_local char g_err[512] = "";
+
+void set_error(const char *fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+}
+
+stream_status cuda_fail(cudaError_t e, const char *what) {
+    set_error("%s: %s", what, cudaGetErrorString(e));
+    return STREAM_ERR_CUDA;
+}
+
+namespace {
+
+long long gcd_ll(long long a, long long b) {
+    while (b) { long long t = a % b; a = b; b = t; }
+    return a;
+}
+
+size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+// Validates *p and fills the kernel-side geometry.
+stream_status make_geom(const stream_problem *p, Geom *g) {
+    if (p == nullptr) { set_error("problem is NULL"); return STREAM_ERR_INVALID_ARG; }
+    if (p->batch < 1 || p->n_q_heads < 1 || p->n_kv_heads < 1 || p->n_q_heads % p->n_kv_heads != 0) {
+        set_error("need batch >= 1 and n_kv_heads dividing n_q_heads (got %d, %d, %d)", p->batch, p->n_q_heads, p->n_kv_heads);
+        return STREAM_ERR_INVALID_ARG;
+    }
+    if (p->T < 1 || p->d < 1 || p->block_q < 1 || p->block_k < 1 || p->k_top < 1) {
+        set_error("T, d, block_q, block_k and k_top must be positive");
+        return STREAM_ERR_INVALID_ARG;
+    }
+    if (p->dtype != STREAM_F32 && p->dtype != STREAM_BF16) { set_error("unknown dtype %d", p->dtype); return STREAM_ERR_INVALID_ARG; }
+    if (p->impl < STREAM_IMPL_AUTO || p->impl > STREAM_IMPL_TENSOR) { set_error("unknown impl %d", p->impl); return STREAM_ERR_INVALID_ARG; }
+    if (p->causal != 0 && p->causal != 1) { set_error("causal must be 0 or 1"); return STREAM_ERR_INVALID_ARG; }
+    if (p->q_stride_t < p->d || p->kv_stride_t < p->d || p->q_stride_h < 0 || p->kv_stride_h < 0 || p->q_stride_b < 0 ||
+        p->kv_stride_b < 0) {
+        set_error("token strides must be >= d and head/batch strides non-negative");
+        return STREAM_ERR_INVALID_ARG;
+    }
+    if (p->k_top > kMaxKTop) { set_error("k_top up to %d (got %d)", kMaxKTop, p->k_top); return STREAM_ERR_UNSUPPORTED; }
+    long long lcm = (long long)p->block_q / gcd_ll(p->block_q, p->block_k) * p->block_k;
+    long long Tp = (p->T + lcm - 1) / lcm * lcm;
+    long long n_qb = (p->T + p->block_q - 1) / p->block_q, N_k = Tp / p->block_k;
+    if (n_qb > 0x7fffffffLL || N_k > 0x7fffffffLL || (long long)p->batch * p->n_q_heads * n_qb > 0x7fffffffLL) {
+        set_error("too many blocks or rows for 32-bit indexing");
+        return STREAM_ERR_UNSUPPORTED;
+    }
+    g->batch = p->batch; g->H = p->n_q_heads; g->G = p->n_kv_heads; g->hpg = p->n_q_heads / p->n_kv_heads;
+    g->T = p->T; g->d = p->d; g->bq = p->block_q; g->bk = p->block_k; g->k_top = p->k_top; g->causal = p->causal;
+    g->n_qb = (int)n_qb; g->N_k = (int)N_k;
+    // levels until every node is a single block: nodes start with at most ceil(N_k / k) blocks and
+    // the larger half of n blocks has ceil(n / 2). With N_k > 1 the first level always runs (it is
+    // where scores are first computed), matching n_it = ceil(log2 N_k) >= 1.
+    long long sz = (N_k + p->k_top - 1) / p->k_top;
+    int levels = 0;
+    while (sz > 1) { sz = (sz + 1) / 2; ++levels; }
+    g->levels = N_k > 1 ? (levels > 1 ? levels : 1) : 0;
+    g->qs_b = p->q_stride_b; g->qs_h = p->q_stride_h; g->qs_t = p->q_stride_t;
+    g->ks_b = p->kv_stride_b; g->ks_h = p->kv_stride_h; g->ks_t = p->kv_stride_t;
+    return STREAM_OK;
+}
+
+size_t elem_size(int dtype) { return dtype == STREAM_F32 ? 4 : 2; }
+
+struct StagingLayout { size_t q, k, v, mask, out, ws, total; };
+
+StagingLayout staging_layout(const stream_problem *p, const Geom &g) {
+    StagingLayout s;
+    size_t e = elem_size(p->dtype);
+    size_t qb = (size_t)g.batch * g.H * g.T * g.d * e, kb = (size_t)g.batch * g.G * g.T * g.d * e;
+    size_t mb = (size_t)g.batch * g.H * g.n_qb * g.k_top * sizeof(int32_t);
+    s.q = 0; s.k = s.q + align256(qb); s.v = s.k + align256(kb); s.mask = s.v + align256(kb);
+    s.out = s.mask + align256(mb); s.ws = s.out + align256(qb); s.total = s.ws + sizeof(WorkspaceHeader);
+    return s;
+}
+
+bool dense_layout(const stream_problem *p) {
+    return p->q_stride_t == p->d && p->q_stride_h == p->T * p->d && p->q_stride_b == (long long)p->n_q_heads * p->T * p->d &&
+           p->kv_stride_t == p->d && p->kv_stride_h == p->T * p->d && p->kv_stride_b == (long long)p->n_kv_heads * p->T * p->d;
+}
+
+}  // namespace
+}  // namespace stream
+
+using namespace stream;
+
+extern "C" {
+
+int stream_version(void) { return 100; }
+
+const char *stream_last_error(void) { return g_err; }
+
+size_t stream_workspace_bytes(const stream_problem *p) {
+    Geom g;
+    if (make_geom(p, &g) != STREAM_OK) return 0;
+    return sizeof(WorkspaceHeader);
+}
+
+stream_status stream_build_mask(const stream_problem *p, const void *q, const void *k, int32_t *mask_out,
+                                float *score_out, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    Geom g;
+    stream_status rc = make_geom(p, &g);
+    if (rc != STREAM_OK) return rc;
+    if (q == nullptr || k == nullptr || mask_out == nullptr) { set_error("q, k and mask_out must not be NULL"); return STREAM_ERR_INVALID_ARG; }
+    if (workspace == nullptr || workspace_bytes < sizeof(WorkspaceHeader) || ((uintptr_t)workspace & 255) != 0) {
+        set_error("workspace must be a 256-byte aligned device buffer of at least %zu bytes", sizeof(WorkspaceHeader));
+        return STREAM_ERR_WORKSPACE;
+    }
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    WorkspaceHeader *ws = (WorkspaceHeader *)workspace;
+    const bool tc_ok = mask_tc_supported(g, p->dtype);
+    if (p->impl == STREAM_IMPL_TENSOR && !tc_ok) {
+        set_error("tensor-core mask kernel needs bf16, d = 128, block_q = block_k = 64, k_top <= 64, causal, 16-byte aligned strides");
+        return STREAM_ERR_UNSUPPORTED;
+    }
+    cudaError_t e = cudaMemsetAsync(ws, 0, sizeof(WorkspaceHeader), st);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(workspace)");
+    if (tc_ok && p->impl != STREAM_IMPL_GENERIC) return launch_mask_tc(g, q, k, mask_out, score_out, ws, st);
+    return launch_mask_generic(g, p->dtype, q, k, mask_out, score_out, ws, st);
+}
+
+stream_status stream_sparse_attention(const stream_problem *p, const void *q, const void *k, const void *v,
+                                      const int32_t *mask, float scale, void *out, void *cuda_stream) {
+    Geom g;
+    stream_status rc = make_geom(p, &g);
+    if (rc != STREAM_OK) return rc;
+    if (q == nullptr || k == nullptr || v == nullptr || mask == nullptr || out == nullptr) {
+        set_error("q, k, v, mask and out must not be NULL");
+        return STREAM_ERR_INVALID_ARG;
+    }
+    if (!(scale > 0.f)) scale = 1.0f / sqrtf((float)g.d);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const bool tc_ok = attn_tc_supported(g, p->dtype);
+    if (p->impl == STREAM_IMPL_TENSOR && !tc_ok) {
+        set_error("tensor-core attention kernel needs bf16, d = 128, block_q = block_k = 64");
+        return STREAM_ERR_UNSUPPORTED;
+    }
+    if (tc_ok && p->impl != STREAM_IMPL_GENERIC) return launch_attn_tc(g, q, k, v, mask, scale, out, st);
+    return launch_attn_generic(g, p->dtype, q, k, v, mask, scale, out, st);
+}
+
+stream_status stream_read_stats(const void *workspace, stream_stats *out, void *cuda_stream) {
+    if (workspace == nullptr || out == nullptr) { set_error("workspace and out must not be NULL"); return STREAM_ERR_INVALID_ARG; }
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaError_t e = cudaMemcpyAsync(out, workspace, sizeof(stream_stats), cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpyAsync(stats)");
+    e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+    if (out->error != 0) {
+        set_error("kernel gave up on a bounded wait: code %u, info %u", out->error, out->error_info);
+        return STREAM_ERR_DEVICE_CHECK;
+    }
+    return STREAM_OK;
+}
+
+size_t stream_host_staging_bytes(const stream_problem *p) {
+    Geom g;
+    if (make_geom(p, &g) != STREAM_OK) return 0;
+    return staging_layout(p, g).total;
+}
+
+stream_status stream_run_host(const stream_problem *p, const void *q_host, const void *k_host, const void *v_host,
+                              int32_t *mask_host, void *out_host, float scale, void *staging,
+                              size_t staging_bytes, void *cuda_stream) {
+    Geom g;
+    stream_status rc = make_geom(p, &g);
+    if (rc != STREAM_OK) return rc;
+    if (!q_host || !k_host || !v_host || !mask_host || !out_host) { set_error("host pointers must not be NULL"); return STREAM_ERR_INVALID_ARG; }
+    if (!dense_layout(p)) { set_error("stream_run_host needs dense [batch, heads, T, d] host tensors"); return STREAM_ERR_INVALID_ARG; }
+    StagingLayout s = staging_layout(p, g);
+    if (staging == nullptr || staging_bytes < s.total || ((uintptr_t)staging & 255) != 0) {
+        set_error("staging must be a 256-byte aligned device buffer of at least %zu bytes", s.total);
+        return STREAM_ERR_WORKSPACE;
+    }
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    char *base = (char *)staging;
+    size_t e = elem_size(p->dtype);
+    size_t qb = (size_t)g.batch * g.H * g.T * g.d * e, kb = (size_t)g.batch * g.G * g.T * g.d * e;
+    size_t mb = (size_t)g.batch * g.H * g.n_qb * g.k_top * sizeof(int32_t);
+    cudaError_t ce;
+    if ((ce = cudaMemcpyAsync(base + s.q, q_host, qb, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(ce, "H2D q");
+    if ((ce = cudaMemcpyAsync(base + s.k, k_host, kb, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(ce, "H2D k");
+    if ((ce = cudaMemcpyAsync(base + s.v, v_host, kb, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(ce, "H2D v");
+    rc = stream_build_mask(p, base + s.q, base + s.k, (int32_t *)(base + s.mask), nullptr, base + s.ws,
+                           sizeof(WorkspaceHeader), cuda_stream);
+    if (rc != STREAM_OK) return rc;
+    rc = stream_sparse_attention(p, base + s.q, base + s.k, base + s.v, (const int32_t *)(base + s.mask), scale,
+                                 base + s.out, cuda_stream);
+    if (rc != STREAM_OK) return rc;
+    if ((ce = cudaMemcpyAsync(mask_host, base + s.mask, mb, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(ce, "D2H mask");
+    if ((ce = cudaMemcpyAsync(out_host, base + s.out, qb, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(ce, "D2H out");
+    return STREAM_OK;
+}
+
+}  // extern "C"

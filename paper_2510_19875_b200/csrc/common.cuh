@@ -1,0 +1,61 @@
+// Shared declarations of the CUDA side of libstream (not shared with the CPU oracle).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "stream.h"
+
+namespace stream {
+
+// Problem geometry as the kernels see it.
+struct Geom {
+    int batch, H, G, hpg;       // heads; hpg = H / G
+    long long T;
+    int d, bq, bk, k_top, causal;
+    int n_qb;                   // ceil(T / bq): rows per head
+    int N_k;                    // key blocks after padding T to a multiple of lcm(bq, bk)
+    int levels;                 // split levels that can change the result
+    long long qs_b, qs_h, qs_t; // element strides
+    long long ks_b, ks_h, ks_t;
+};
+
+// Header at the start of the mask workspace. The first 24 bytes mirror stream_stats.
+struct WorkspaceHeader {
+    unsigned long long tiles_scored;
+    unsigned long long rows;
+    unsigned int error;
+    unsigned int error_info;
+    unsigned int work_counter;  // next work item of the persistent kernels
+    unsigned int pad[57];
+};
+static_assert(sizeof(WorkspaceHeader) == 256, "workspace header is 256 bytes");
+
+constexpr int kMaxKTop = 1024;
+
+void set_error(const char *fmt, ...);
+stream_status cuda_fail(cudaError_t e, const char *what);
+
+// Launchers (each validates what only it can support and returns UNSUPPORTED otherwise).
+stream_status launch_mask_generic(const Geom &g, int dtype, const void *q, const void *k, int32_t *mask,
+                                  float *score, WorkspaceHeader *ws, cudaStream_t st);
+stream_status launch_attn_generic(const Geom &g, int dtype, const void *q, const void *k, const void *v,
+                                  const int32_t *mask, float scale, void *out, cudaStream_t st);
+bool mask_tc_supported(const Geom &g, int dtype);
+stream_status launch_mask_tc(const Geom &g, const void *q, const void *k, int32_t *mask, float *score,
+                             WorkspaceHeader *ws, cudaStream_t st);
+bool attn_tc_supported(const Geom &g, int dtype);
+stream_status launch_attn_tc(const Geom &g, const void *q, const void *k, const void *v, const int32_t *mask,
+                             float scale, void *out, cudaStream_t st);
+
+__device__ __forceinline__ float to_float(float x) { return x; }
+__device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+// Last key block a row may look at (C^blk of Algorithm 2 in closed form), -1 if none.
+__host__ __device__ inline int last_valid_block(const Geom &g, int qb) {
+    long long last_tok = g.causal ? ((long long)qb * g.bq + g.bq - 1) : (g.T - 1);
+    if (last_tok > g.T - 1) last_tok = g.T - 1;
+    return (int)(last_tok / g.bk);
+}
+
+}  // namespace stream

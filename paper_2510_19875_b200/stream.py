@@ -1,0 +1,227 @@
+"""Python binding of libstream (argument marshalling only; every step runs in the CUDA library).
+
+The ``stream_*`` functions mirror the C ABI in ``include/stream.h`` one to one and take torch
+CUDA tensors (or raw integer addresses) where the C side takes device pointers. ``build_mask``,
+``sparse_attention`` and ``run_host`` are conveniences that allocate outputs with torch and fill
+in the problem struct from tensor shapes and strides. PyTorch is used for device memory and
+streams only.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libstream.so")
+
+STREAM_OK, STREAM_ERR_INVALID_ARG, STREAM_ERR_UNSUPPORTED, STREAM_ERR_WORKSPACE, STREAM_ERR_CUDA, STREAM_ERR_DEVICE_CHECK = range(6)
+STREAM_F32, STREAM_BF16 = 0, 1
+IMPL = {"auto": 0, "generic": 1, "tensor": 2}
+_STATUS_NAMES = ["OK", "INVALID_ARG", "UNSUPPORTED", "WORKSPACE", "CUDA", "DEVICE_CHECK"]
+
+
+class StreamProblem(ctypes.Structure):
+    """``stream_problem`` of stream.h."""
+
+    _fields_ = [
+        ("batch", ctypes.c_int32), ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
+        ("T", ctypes.c_int64),
+        ("d", ctypes.c_int32), ("block_q", ctypes.c_int32), ("block_k", ctypes.c_int32), ("k_top", ctypes.c_int32),
+        ("causal", ctypes.c_int32), ("dtype", ctypes.c_int32), ("impl", ctypes.c_int32),
+        ("q_stride_b", ctypes.c_int64), ("q_stride_h", ctypes.c_int64), ("q_stride_t", ctypes.c_int64),
+        ("kv_stride_b", ctypes.c_int64), ("kv_stride_h", ctypes.c_int64), ("kv_stride_t", ctypes.c_int64),
+    ]
+
+
+class StreamStats(ctypes.Structure):
+    """``stream_stats`` of stream.h."""
+
+    _fields_ = [("tiles_scored", ctypes.c_uint64), ("rows", ctypes.c_uint64), ("error", ctypes.c_uint32),
+                ("error_info", ctypes.c_uint32)]
+
+
+class StreamError(RuntimeError):
+    def __init__(self, status: int, text: str):
+        super().__init__(f"libstream: STREAM_ERR_{_STATUS_NAMES[status]}: {text}")
+        self.status = status
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def _load():
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise RuntimeError(
+            f"{_LIB_PATH} is missing: build it with `python -m paper_2510_19875_b200.build` "
+            "(there is no fallback path without the CUDA library)")
+    lib = ctypes.CDLL(_LIB_PATH)
+    P, vp, sz = ctypes.POINTER(StreamProblem), ctypes.c_void_p, ctypes.c_size_t
+    lib.stream_version.restype = ctypes.c_int
+    lib.stream_version.argtypes = []
+    lib.stream_last_error.restype = ctypes.c_char_p
+    lib.stream_last_error.argtypes = []
+    lib.stream_workspace_bytes.restype = sz
+    lib.stream_workspace_bytes.argtypes = [P]
+    lib.stream_build_mask.restype = ctypes.c_int
+    lib.stream_build_mask.argtypes = [P, vp, vp, vp, vp, vp, sz, vp]
+    lib.stream_sparse_attention.restype = ctypes.c_int
+    lib.stream_sparse_attention.argtypes = [P, vp, vp, vp, vp, ctypes.c_float, vp, vp]
+    lib.stream_read_stats.restype = ctypes.c_int
+    lib.stream_read_stats.argtypes = [vp, ctypes.POINTER(StreamStats), vp]
+    lib.stream_host_staging_bytes.restype = sz
+    lib.stream_host_staging_bytes.argtypes = [P]
+    lib.stream_run_host.restype = ctypes.c_int
+    lib.stream_run_host.argtypes = [P, vp, vp, vp, vp, vp, ctypes.c_float, vp, sz, vp]
+    _lib = lib
+    return lib
+
+
+def _addr(x):
+    if x is None:
+        return None
+    if isinstance(x, torch.Tensor):
+        return x.data_ptr()
+    return int(x)
+
+
+def _stream_handle(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if isinstance(stream, torch.cuda.Stream) else int(stream)
+
+
+def _raise(status: int):
+    if status != STREAM_OK:
+        raise StreamError(status, _load().stream_last_error().decode())
+
+
+# ----------------------------------------------------------------------------------------------
+# One-to-one with the C ABI
+# ----------------------------------------------------------------------------------------------
+def stream_version() -> int:
+    return int(_load().stream_version())
+
+
+def stream_last_error() -> str:
+    return _load().stream_last_error().decode()
+
+
+def stream_workspace_bytes(p: StreamProblem) -> int:
+    return int(_load().stream_workspace_bytes(ctypes.byref(p)))
+
+
+def stream_build_mask(p: StreamProblem, q, k, mask_out, score_out, workspace, workspace_bytes: int, stream=None) -> None:
+    _raise(_load().stream_build_mask(ctypes.byref(p), _addr(q), _addr(k), _addr(mask_out), _addr(score_out),
+                                     _addr(workspace), workspace_bytes, _stream_handle(stream)))
+
+
+def stream_sparse_attention(p: StreamProblem, q, k, v, mask, scale: float, out, stream=None) -> None:
+    _raise(_load().stream_sparse_attention(ctypes.byref(p), _addr(q), _addr(k), _addr(v), _addr(mask), float(scale),
+                                           _addr(out), _stream_handle(stream)))
+
+
+def stream_read_stats(workspace, stream=None) -> StreamStats:
+    st = StreamStats()
+    _raise(_load().stream_read_stats(_addr(workspace), ctypes.byref(st), _stream_handle(stream)))
+    return st
+
+
+def stream_host_staging_bytes(p: StreamProblem) -> int:
+    return int(_load().stream_host_staging_bytes(ctypes.byref(p)))
+
+
+def stream_run_host(p: StreamProblem, q_host, k_host, v_host, mask_host, out_host, scale: float, staging,
+                    staging_bytes: int, stream=None) -> None:
+    _raise(_load().stream_run_host(ctypes.byref(p), _addr(q_host), _addr(k_host), _addr(v_host), _addr(mask_host),
+                                   _addr(out_host), float(scale), _addr(staging), staging_bytes, _stream_handle(stream)))
+
+
+# ----------------------------------------------------------------------------------------------
+# Conveniences: problem struct from tensors, outputs allocated with torch
+# ----------------------------------------------------------------------------------------------
+def make_problem(q: torch.Tensor, k: torch.Tensor, *, block_q: int, block_k: int, k_top: int, causal: bool = True,
+                 impl: str = "auto") -> StreamProblem:
+    """Problem struct for q ``[B, H, T, d]`` and k ``[B, G, T, d]`` (any strides with unit innermost)."""
+    if q.dim() != 4 or k.dim() != 4 or q.shape[0] != k.shape[0] or q.shape[2:] != k.shape[2:]:
+        raise ValueError("q must be [B, H, T, d] and k [B, G, T, d] with matching B, T, d")
+    if q.dtype != k.dtype or q.dtype not in (torch.float32, torch.bfloat16):
+        raise ValueError("q and k must both be float32 or bfloat16")
+    if q.stride(3) != 1 or k.stride(3) != 1:
+        raise ValueError("innermost stride must be 1")
+    B, H, T, d = q.shape
+    return StreamProblem(B, H, k.shape[1], T, d, block_q, block_k, k_top, int(causal),
+                         STREAM_F32 if q.dtype == torch.float32 else STREAM_BF16, IMPL[impl],
+                         q.stride(0), q.stride(1), q.stride(2), k.stride(0), k.stride(1), k.stride(2))
+
+
+def n_query_blocks(p: StreamProblem) -> int:
+    return -(-p.T // p.block_q)
+
+
+@dataclass
+class MaskResult:
+    mask: torch.Tensor            # int32 [B, H, n_query_blocks, k_top]
+    scores: torch.Tensor | None   # float32, same shape, if requested
+    workspace: torch.Tensor       # holds the counters of this call; see stream_read_stats
+
+    def stats(self, stream=None) -> StreamStats:
+        return stream_read_stats(self.workspace, stream)
+
+
+def new_workspace(p: StreamProblem, device) -> torch.Tensor:
+    n = stream_workspace_bytes(p)
+    if n == 0:
+        raise StreamError(STREAM_ERR_INVALID_ARG, stream_last_error())
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def build_mask(q: torch.Tensor, k: torch.Tensor, *, block_q: int, block_k: int, k_top: int, causal: bool = True,
+               impl: str = "auto", want_scores: bool = False, mask_out: torch.Tensor | None = None,
+               workspace: torch.Tensor | None = None, stream=None) -> MaskResult:
+    if not q.is_cuda or not k.is_cuda:
+        raise ValueError("q and k must be CUDA tensors (there is no CPU path)")
+    p = make_problem(q, k, block_q=block_q, block_k=block_k, k_top=k_top, causal=causal, impl=impl)
+    shape = (p.batch, p.n_q_heads, n_query_blocks(p), k_top)
+    mask = mask_out if mask_out is not None else torch.empty(shape, dtype=torch.int32, device=q.device)
+    scores = torch.empty(shape, dtype=torch.float32, device=q.device) if want_scores else None
+    ws = workspace if workspace is not None else new_workspace(p, q.device)
+    stream_build_mask(p, q, k, mask, scores, ws, ws.numel(), stream)
+    return MaskResult(mask, scores, ws)
+
+
+def sparse_attention(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, mask: torch.Tensor, *, block_q: int,
+                     block_k: int, causal: bool = True, scale: float = 0.0, impl: str = "auto",
+                     out: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    if not (q.is_cuda and k.is_cuda and v.is_cuda and mask.is_cuda):
+        raise ValueError("q, k, v and mask must be CUDA tensors (there is no CPU path)")
+    if v.shape != k.shape or v.stride() != k.stride() or v.dtype != k.dtype:
+        raise ValueError("v must have k's shape, strides and dtype")
+    if mask.dtype != torch.int32 or not mask.is_contiguous():
+        raise ValueError("mask must be a contiguous int32 tensor")
+    p = make_problem(q, k, block_q=block_q, block_k=block_k, k_top=mask.shape[-1], causal=causal, impl=impl)
+    if tuple(mask.shape) != (p.batch, p.n_q_heads, n_query_blocks(p), mask.shape[-1]):
+        raise ValueError("mask must be [B, H, ceil(T / block_q), k_top]")
+    if out is None:
+        out = torch.empty((p.batch, p.n_q_heads, p.T, p.d), dtype=q.dtype, device=q.device)
+    stream_sparse_attention(p, q, k, v, mask, scale, out, stream)
+    return out
+
+
+def run_host(q_host: torch.Tensor, k_host: torch.Tensor, v_host: torch.Tensor, mask_host: torch.Tensor,
+             out_host: torch.Tensor, staging: torch.Tensor, *, block_q: int, block_k: int, k_top: int,
+             causal: bool = True, scale: float = 0.0, impl: str = "auto", stream=None) -> None:
+    """Whole path from (pinned) host tensors through a caller-provided device staging buffer."""
+    if q_host.is_cuda or not staging.is_cuda:
+        raise ValueError("q/k/v/mask/out live on the host, staging on the device")
+    p = make_problem(q_host, k_host, block_q=block_q, block_k=block_k, k_top=k_top, causal=causal, impl=impl)
+    stream_run_host(p, q_host, k_host, v_host, mask_host, out_host, scale, staging, staging.numel(), stream)

@@ -19,6 +19,8 @@ Structure (all optional, combined per workload):
 """
 from __future__ import annotations
 
+import os
+from concurrent.futures import ThreadPoolExecutor
 from dataclasses import dataclass, field, replace
 
 import numpy as np
@@ -123,50 +125,59 @@ def generate(spec: WorkloadSpec, with_v: bool = True) -> Workload:
     cast = (lambda a: a) if spec.dtype == "f32" else to_bf16_bits
     notes: dict = {}
     n_blocks = spec.n_blocks
-    for b in range(B):
+    def fill_group(b: int, g: int) -> None:
         seed = spec.seed + b  # stacks: one independent seed per layer
-        for g in range(G):
-            aux = _rng(seed, _AUX, 0, g)
-            kg = _rng(seed, _K, 0, g).standard_normal((T, d), dtype=np.float32)
-            sink_u = _unit(aux.standard_normal(d).astype(np.float32)) if spec.sink else None
-            win = None
+        aux = _rng(seed, _AUX, 0, g)
+        kg = _rng(seed, _K, 0, g).standard_normal((T, d), dtype=np.float32)
+        sink_u = _unit(aux.standard_normal(d).astype(np.float32)) if spec.sink else None
+        win = None
+        if spec.local:
+            n_win = -(-T // 256)
+            win = aux.standard_normal((n_win, d)).astype(np.float32)
+            kg += 0.5 * win[np.arange(T) // 256]
+        if spec.sink:
+            kg[0] = 4.0 * np.sqrt(np.float32(d)) * sink_u
+        anchor_pos = None
+        if spec.anchors:
+            n_anchor = min(64, T - 1)
+            anchor_pos = np.sort(aux.choice(np.arange(1, T), size=n_anchor, replace=False))
+            notes[("anchors", b, g)] = anchor_pos
+        needle_dir = None
+        if spec.needle:
+            blk = int(aux.integers(1, max(2, n_blocks // 2)))
+            needle_dir = _unit(aux.standard_normal(d).astype(np.float32))
+            lo, hi = blk * spec.block, min(T, (blk + 1) * spec.block)
+            kg[lo:hi] = np.linalg.norm(kg[lo:hi], axis=-1, keepdims=True) * needle_dir
+            notes[("needle_block", b, g)] = blk
+        k[b, g] = cast(kg)
+        if with_v:
+            v[b, g] = cast(_rng(seed, _V, 0, g).standard_normal((T, d), dtype=np.float32))
+        for h in range(g * hpg, (g + 1) * hpg):
+            qh = _rng(seed, _Q, 0, h).standard_normal((T, d), dtype=np.float32)
             if spec.local:
-                n_win = -(-T // 256)
-                win = aux.standard_normal((n_win, d)).astype(np.float32)
-                kg += 0.5 * win[np.arange(T) // 256]
+                qh += win[np.arange(T) // 256]
             if spec.sink:
-                kg[0] = 4.0 * np.sqrt(np.float32(d)) * sink_u
-            anchor_pos = None
+                qh += 2.0 * sink_u
             if spec.anchors:
-                n_anchor = min(64, T - 1)
-                anchor_pos = np.sort(aux.choice(np.arange(1, T), size=n_anchor, replace=False))
-                notes[("anchors", b, g)] = anchor_pos
-            needle_dir = None
+                hr = _rng(seed, _AUX, 1, h)
+                chosen = np.nonzero(hr.random(T) < 0.1)[0]
+                before = np.searchsorted(anchor_pos, chosen, side="left")  # anchors strictly before t
+                chosen, before = chosen[before > 0], before[before > 0]
+                pick = np.minimum((hr.random(chosen.shape[0]) * before).astype(np.int64), before - 1)
+                target = _unit(kg[anchor_pos[pick]])
+                qh[chosen] = _rotate_towards(qh[chosen], target, 0.8)
             if spec.needle:
-                blk = int(aux.integers(1, max(2, n_blocks // 2)))
-                needle_dir = _unit(aux.standard_normal(d).astype(np.float32))
-                lo, hi = blk * spec.block, min(T, (blk + 1) * spec.block)
-                kg[lo:hi] = np.linalg.norm(kg[lo:hi], axis=-1, keepdims=True) * needle_dir
-                notes[("needle_block", b, g)] = blk
-            k[b, g] = cast(kg)
-            if with_v:
-                v[b, g] = cast(_rng(seed, _V, 0, g).standard_normal((T, d), dtype=np.float32))
-            for h in range(g * hpg, (g + 1) * hpg):
-                qh = _rng(seed, _Q, 0, h).standard_normal((T, d), dtype=np.float32)
-                if spec.local:
-                    qh += win[np.arange(T) // 256]
-                if spec.sink:
-                    qh += 2.0 * sink_u
-                if spec.anchors:
-                    hr = _rng(seed, _AUX, 1, h)
-                    chosen = np.nonzero(hr.random(T) < 0.1)[0]
-                    before = np.searchsorted(anchor_pos, chosen, side="left")  # anchors strictly before t
-                    chosen, before = chosen[before > 0], before[before > 0]
-                    pick = np.minimum((hr.random(chosen.shape[0]) * before).astype(np.int64), before - 1)
-                    target = _unit(kg[anchor_pos[pick]])
-                    qh[chosen] = _rotate_towards(qh[chosen], target, 0.8)
-                if spec.needle:
-                    lo = max(0, T - 128)
-                    qh[lo:] = _rotate_towards(qh[lo:], needle_dir, 0.9)
-                q[b, h] = cast(qh)
+                lo = max(0, T - 128)
+                qh[lo:] = _rotate_towards(qh[lo:], needle_dir, 0.9)
+            q[b, h] = cast(qh)
+
+    # kv groups are independent streams: fill them on a few threads (numpy releases the GIL)
+    groups = [(b, g) for b in range(B) for g in range(G)]
+    n_workers = max(1, min(len(groups), os.cpu_count() or 1, 16))
+    if n_workers == 1:
+        for bg in groups:
+            fill_group(*bg)
+    else:
+        with ThreadPoolExecutor(n_workers) as pool:
+            list(pool.map(lambda bg: fill_group(*bg), groups))
     return Workload(spec, q, k, v, notes)

@@ -1,0 +1,107 @@
+"""Host-side checks that need no GPU: the library loads, exports what the header declares, and
+rejects bad arguments before anything is launched."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2510_19875_b200 import build as stream_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def S():
+    stream_build.build_library()
+    from paper_2510_19875_b200 import stream
+
+    return stream
+
+
+def declared_functions():
+    names = []
+    inc = os.path.join(ROOT, "include")
+    for fn in sorted(os.listdir(inc)):
+        text = open(os.path.join(inc, fn)).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        names += re.findall(r"\b(stream_[a-z_0-9]+)\s*\(", text)
+    return sorted(set(names))
+
+
+def test_library_exports_every_declared_symbol(S):
+    lib = ctypes.CDLL(S.library_path())
+    names = declared_functions()
+    assert {"stream_build_mask", "stream_sparse_attention", "stream_workspace_bytes", "stream_run_host",
+            "stream_host_staging_bytes", "stream_read_stats", "stream_last_error", "stream_version"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), n
+        assert hasattr(S, n), f"binding lacks {n}"
+    assert S.stream_version() >= 100
+
+
+def good_problem(S, **kw):
+    base = dict(batch=1, n_q_heads=4, n_kv_heads=2, T=256, d=128, block_q=64, block_k=64, k_top=4, causal=1,
+                dtype=S.STREAM_BF16, impl=0, q_stride_b=4 * 256 * 128, q_stride_h=256 * 128, q_stride_t=128,
+                kv_stride_b=2 * 256 * 128, kv_stride_h=256 * 128, kv_stride_t=128)
+    base.update(kw)
+    return S.StreamProblem(**base)
+
+
+@pytest.mark.parametrize("kw", [
+    dict(batch=0), dict(n_kv_heads=3), dict(T=0), dict(d=0), dict(block_q=0), dict(block_k=-1), dict(k_top=0),
+    dict(dtype=7), dict(impl=9), dict(causal=2), dict(q_stride_t=64), dict(kv_stride_h=-1),
+])
+def test_invalid_problem_is_rejected_on_the_host(S, kw):
+    p = good_problem(S, **kw)
+    assert S.stream_workspace_bytes(p) == 0
+    assert S.stream_host_staging_bytes(p) == 0
+    with pytest.raises(S.StreamError) as e:
+        S.stream_build_mask(p, 256, 256, 256, None, 256, 256, stream=0)
+    assert e.value.status == S.STREAM_ERR_INVALID_ARG
+    assert S.stream_last_error() != ""
+
+
+def test_null_pointers_and_workspace_are_checked_before_launch(S):
+    p = good_problem(S)
+    assert S.stream_workspace_bytes(p) >= 256
+    with pytest.raises(S.StreamError) as e:
+        S.stream_build_mask(p, None, 256, 256, None, 256, 256, stream=0)
+    assert e.value.status == S.STREAM_ERR_INVALID_ARG
+    for ws, nbytes in ((None, 256), (256, 8), (264, 4096)):  # missing, too small, misaligned
+        with pytest.raises(S.StreamError) as e:
+            S.stream_build_mask(p, 256, 256, 256, None, ws, nbytes, stream=0)
+        assert e.value.status == S.STREAM_ERR_WORKSPACE
+    with pytest.raises(S.StreamError) as e:
+        S.stream_sparse_attention(p, 256, 256, None, 256, 0.0, 256, stream=0)
+    assert e.value.status == S.STREAM_ERR_INVALID_ARG
+    with pytest.raises(S.StreamError) as e:
+        S.stream_run_host(p, 256, 256, 256, 256, 256, 0.0, None, 0, stream=0)
+    assert e.value.status == S.STREAM_ERR_WORKSPACE
+
+
+def test_unsupported_shapes_say_so(S):
+    with pytest.raises(S.StreamError) as e:
+        S.stream_build_mask(good_problem(S, k_top=5000), 256, 256, 256, None, 256, 256, stream=0)
+    assert e.value.status == S.STREAM_ERR_UNSUPPORTED
+    # the tensor-core kernels take one shape only; asking for them elsewhere is an error, not a fallback
+    with pytest.raises(S.StreamError) as e:
+        S.stream_build_mask(good_problem(S, dtype=S.STREAM_F32, impl=2), 256, 256, 256, None, 256, 256, stream=0)
+    assert e.value.status == S.STREAM_ERR_UNSUPPORTED
+
+
+def test_cpu_tensors_are_refused(S):
+    import torch
+
+    q = torch.zeros(1, 1, 64, 64)
+    with pytest.raises(ValueError):
+        S.build_mask(q, q, block_q=32, block_k=32, k_top=2)
+    with pytest.raises(ValueError):
+        S.sparse_attention(q, q, q, torch.zeros(1, 1, 2, 2, dtype=torch.int32), block_q=32, block_k=32)
+
+
+def test_staging_size_covers_all_buffers(S):
+    p = good_problem(S)
+    e = 2
+    need = (4 * 256 * 128 * e) * 2 + (2 * 256 * 128 * e) * 2 + 4 * 4 * 4 * 4 + 256
+    assert S.stream_host_staging_bytes(p) >= need

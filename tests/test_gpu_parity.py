@@ -1,0 +1,187 @@
+"""GPU parity: the CUDA library against the CPU oracle on the same seeded inputs, through the
+C ABI. Masks must be bit-exact except rows the oracle flags as ties (k-th / (k+1)-th score gap
+below 1e-5 relative), which are counted; attention must stay within 2e-2 (bf16) / 1e-4 (fp32)."""
+import numpy as np
+import pytest
+import torch
+
+from helpers import check_mask_invariants, compare_masks, oracle_problem, sample_rows
+from oracle import stream_oracle as so
+from paper_2510_19875_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+ATTN_TOL = {"bf16": 2e-2, "f32": 1e-4}
+
+
+@pytest.fixture(scope="module")
+def S():
+    from paper_2510_19875_b200 import stream
+
+    assert stream.stream_version() >= 100
+    return stream
+
+
+def run_mask(S, w, *, impl="auto", block_q=None, block_k=None, k_top=None, causal=True, want_scores=False):
+    spec = w.spec
+    q, k, _ = w.torch_tensors("cuda")
+    res = S.build_mask(q, k, block_q=block_q or spec.block, block_k=block_k or spec.block,
+                       k_top=k_top or spec.k_top, causal=causal, impl=impl, want_scores=want_scores)
+    torch.cuda.synchronize()
+    return res
+
+
+def assert_mask_parity(S, w, rows, *, impl="auto", score_cache=True, **kw):
+    spec = w.spec
+    res = run_mask(S, w, impl=impl, want_scores=True, **kw)
+    mask = res.mask.cpu().numpy()
+    check_mask_invariants(mask, spec, block_q=kw.get("block_q"), block_k=kw.get("block_k"), causal=kw.get("causal", True))
+    p = oracle_problem(spec, **kw)
+    ora = so.build_mask_rows(p, w.q, w.k, rows, score_cache=score_cache, want_scores=True)
+    flat = mask.reshape(-1, mask.shape[-1])
+    got = flat if rows is None else flat[rows]
+    report = compare_masks(got, ora)
+    assert report["bad"] == 0, report
+    # scores of kept blocks: fp32 accumulation on the GPU against fp64-then-round in the oracle
+    sc = res.scores.cpu().numpy().reshape(-1, mask.shape[-1])
+    sc = sc if rows is None else sc[rows]
+    same = (got == ora["mask"]).all(axis=1)
+    fin = np.isfinite(ora["scores"][same])
+    np.testing.assert_allclose(sc[same][fin], ora["scores"][same][fin], rtol=2e-5, atol=2e-5)
+    assert (sc[same][~fin] == -np.inf).all()
+    st = res.stats()
+    assert st.rows == flat.shape[0] and st.error == 0
+    if rows is None:
+        agree = same & (ora["min_gap"] >= 1e-5)
+        if agree.all():
+            assert st.tiles_scored == int(ora["tiles"].sum())
+    return report
+
+
+def small_spec(**kw):
+    base = dict(name="t", seed=5, batch=1, n_q_heads=2, n_kv_heads=1, T=512, d=64, block=32, k_top=4, dtype="f32")
+    base.update(kw)
+    return wl.WorkloadSpec(**base)
+
+
+GENERIC_CASES = [
+    dict(),                                                        # fp32, two levels
+    dict(dtype="bf16", d=128, block=64, T=2048, k_top=8, n_q_heads=4, n_kv_heads=2, sink=True),
+    dict(T=1000, k_top=5),                                         # ragged T, odd k
+    dict(T=777, d=32, block=16, k_top=3, batch=2),                 # batch, ragged, uneven nodes
+    dict(T=512, d=16, block=8, k_top=7, dtype="bf16"),
+    dict(T=256, k_top=16),                                         # k > N_k: full mask, no levels
+    dict(T=64, block=64, k_top=2),                                 # a single key block
+    dict(T=1, block=32, k_top=1, n_q_heads=1),                     # one token
+    dict(T=4096, d=64, block=32, k_top=1, n_q_heads=1),            # k = 1: pure binary descent
+]
+
+
+@pytest.mark.parametrize("kw", GENERIC_CASES)
+def test_mask_generic_small(S, kw):
+    w = wl.generate(small_spec(**kw))
+    assert_mask_parity(S, w, None, impl="generic", score_cache=False)
+
+
+@pytest.mark.parametrize("bq,bk", [(16, 32), (32, 8), (1, 16), (24, 16)])
+def test_mask_generic_unequal_blocks(S, bq, bk):
+    w = wl.generate(small_spec(T=700, k_top=5))
+    assert_mask_parity(S, w, None, impl="generic", score_cache=False, block_q=bq, block_k=bk)
+
+
+def test_mask_generic_non_causal(S):
+    w = wl.generate(small_spec(T=900, k_top=6, n_q_heads=2, n_kv_heads=2))
+    assert_mask_parity(S, w, None, impl="generic", score_cache=False, causal=False)
+
+
+def test_mask_strided_inputs(S):
+    """[B, T, H, d] storage seen through [B, H, T, d] strides gives the same mask."""
+    w = wl.generate(small_spec(dtype="bf16", d=128, block=64, T=1024, k_top=4, n_q_heads=4, n_kv_heads=2))
+    q, k, _ = w.torch_tensors("cuda")
+    ref = S.build_mask(q, k, block_q=64, block_k=64, k_top=4).mask
+    qs = q.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    ks = k.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    assert not qs.is_contiguous()
+    for impl in ("generic", "auto"):
+        got = S.build_mask(qs, ks, block_q=64, block_k=64, k_top=4, impl=impl).mask
+        assert torch.equal(got, ref)
+
+
+def test_config1_single_head_fp32_all_rows(S):
+    w = wl.generate(wl.SPECS["single_head_fp32"])
+    rep = assert_mask_parity(S, w, None, score_cache=False)
+    assert rep["rows"] == 64
+
+
+def attention_parity(S, w, rows, *, impl="auto", block_q=None, block_k=None, causal=True, k_top=None):
+    """Both sides use the ORACLE's mask, so mask tie exemptions cannot leak into this check."""
+    spec = w.spec
+    p = oracle_problem(spec, block_q=block_q, block_k=block_k, causal=causal, k_top=k_top)
+    bq, bk = p.block_q, p.block_k
+    ora_all = so.build_mask_rows(p, w.q, w.k, rows, score_cache=True)
+    nqb = so.num_query_blocks(p)
+    full = np.full((spec.batch * spec.n_q_heads * nqb, p.k_top), -1, np.int32)
+    idx = np.arange(full.shape[0]) if rows is None else rows
+    full[idx] = ora_all["mask"]
+    q, k, v = w.torch_tensors("cuda")
+    mask_dev = torch.from_numpy(full.reshape(spec.batch, spec.n_q_heads, nqb, p.k_top)).cuda()
+    out = S.sparse_attention(q, k, v, mask_dev, block_q=bq, block_k=bk, causal=causal, impl=impl)
+    torch.cuda.synchronize()
+    ref = so.sparse_attention_rows(p, w.q, w.k, w.v, ora_all["mask"], rows)  # [n, bq, d] fp64
+    got = out.float().cpu().numpy().reshape(spec.batch * spec.n_q_heads, spec.T, spec.d)
+    worst = 0.0
+    for i, rid in enumerate(idx):
+        bh, qb = divmod(int(rid), nqb)
+        lo, hi = qb * bq, min(spec.T, qb * bq + bq)
+        worst = max(worst, float(np.abs(got[bh, lo:hi] - ref[i, : hi - lo]).max()))
+    assert worst <= ATTN_TOL[spec.dtype], worst
+    return worst
+
+
+@pytest.mark.parametrize("kw", [
+    dict(),
+    dict(dtype="bf16", d=128, block=64, T=2048, k_top=8, n_q_heads=4, n_kv_heads=2, sink=True),
+    dict(T=777, d=32, block=16, k_top=3, batch=2),
+    dict(T=256, k_top=16),
+])
+def test_attention_generic_small(S, kw):
+    w = wl.generate(small_spec(**kw))
+    attention_parity(S, w, None, impl="generic")
+
+
+def test_attention_generic_unequal_blocks_and_non_causal(S):
+    w = wl.generate(small_spec(T=700, k_top=5))
+    attention_parity(S, w, None, impl="generic", block_q=24, block_k=16)
+    attention_parity(S, w, None, impl="generic", causal=False)
+
+
+def test_full_mask_attention_equals_dense_softmax_attention(S):
+    """k covers every causal block: the sparse pass must reproduce dense causal attention."""
+    w = wl.generate(small_spec(dtype="bf16", d=128, block=64, T=1024, k_top=16, n_q_heads=4, n_kv_heads=2))
+    q, k, v = w.torch_tensors("cuda")
+    res = S.build_mask(q, k, block_q=64, block_k=64, k_top=16)
+    out = S.sparse_attention(q, k, v, res.mask, block_q=64, block_k=64)
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        q.double().cpu(), k.double().cpu().repeat_interleave(2, 1), v.double().cpu().repeat_interleave(2, 1), is_causal=True)
+    assert (out.double().cpu() - ref).abs().max().item() <= 2e-2
+
+
+def test_config1_attention(S):
+    w = wl.generate(wl.SPECS["single_head_fp32"])
+    attention_parity(S, w, None)
+
+
+def test_run_host_matches_device_calls(S):
+    w = wl.generate(small_spec(dtype="bf16", d=128, block=64, T=2048, k_top=8, n_q_heads=4, n_kv_heads=2, sink=True))
+    qh, kh, vh = w.torch_tensors("cpu", pin=True)
+    q, k, v = qh.cuda(), kh.cuda(), vh.cuda()
+    ref = S.build_mask(q, k, block_q=64, block_k=64, k_top=8)
+    out_ref = S.sparse_attention(q, k, v, ref.mask, block_q=64, block_k=64)
+    p = S.make_problem(qh, kh, block_q=64, block_k=64, k_top=8)
+    staging = torch.empty(S.stream_host_staging_bytes(p), dtype=torch.uint8, device="cuda")
+    mask_host = torch.empty(ref.mask.shape, dtype=torch.int32).pin_memory()
+    out_host = torch.empty(out_ref.shape, dtype=out_ref.dtype).pin_memory()
+    S.run_host(qh, kh, vh, mask_host, out_host, staging, block_q=64, block_k=64, k_top=8)
+    torch.cuda.synchronize()
+    assert torch.equal(mask_host, ref.mask.cpu())
+    assert torch.equal(out_host, out_ref.cpu())

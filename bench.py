@@ -1,0 +1,346 @@
+"""Benchmark of the Stream hot path (mask build + block-sparse attention) on synthetic inputs.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+One step = one pass of the whole path over one layer-shaped batch: stream_build_mask followed by
+stream_sparse_attention. The headline workload is the 128k-token chain-of-thought-shaped layer
+(32 query / 8 kv heads, d = 128, bf16, block 64, k = 32). Prints ONE JSON line (rank 0).
+
+N > 1 (under torchrun): every rank processes its own independent layer (different seed); there is
+no data-path collective, so scaling is weak and the value is the sum over ranks divided by the
+slowest rank's time.
+
+``--impl reference`` times the CPU oracle (the plain definition the library is tested against) on
+the host cores, on a bounded sample of rows per step.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "stream_query_token_heads_per_s"
+UNIT = "query-token-heads/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cot_layer_128k")
+    ap.add_argument("--T", type=int, default=0, help="override the workload's context length")
+    ap.add_argument("--kernels", default="auto", choices=["auto", "generic", "tensor"], help="library kernel choice")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0, help="target CPU time of the oracle sample")
+    return ap.parse_args()
+
+
+def get_spec(args, rank=0):
+    from paper_2510_19875_b200 import workloads as wl
+
+    spec = wl.SPECS[args.workload]
+    if args.T:
+        spec = spec.scaled(T=args.T)
+    if rank:
+        spec = spec.scaled(seed=spec.seed + 1000 * rank)
+    return spec
+
+
+def workload_config(spec, extra=None):
+    cfg = {
+        "workload": spec.name, "batch": spec.batch, "n_q_heads": spec.n_q_heads, "n_kv_heads": spec.n_kv_heads,
+        "T": spec.T, "head_dim": spec.d, "block_q": spec.block, "block_k": spec.block, "k_top": spec.k_top,
+        "causal": True, "seed": spec.seed,
+        "structure": [n for n in ("sink", "local", "anchors", "needle") if getattr(spec, n)],
+    }
+    cfg.update(extra or {})
+    return cfg
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons, sampled every 200 ms while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.lines, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "200"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._pump, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])), mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    except (OSError, KeyError, ValueError):
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def ncu_traffic(kernel_key: str, units: int):
+    """DRAM bytes per launch from the committed ncu summary, scaled by the units processed."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    try:
+        with open(path) as fh:
+            rec = json.load(fh)[kernel_key]
+        return rec["dram_bytes_per_unit"] * units
+    except (OSError, KeyError, ValueError):
+        return None
+
+
+def oracle_sample_rate(spec, w, seconds: float):
+    """Times the oracle (mask rows + attention rows, literal mode) on a seeded row sample sized for
+    about `seconds` of wall time; returns (query-token-heads/s, threads, description)."""
+    import numpy as np
+
+    from oracle import stream_oracle as so
+
+    p = so.OracleProblem(spec.batch, spec.n_q_heads, spec.n_kv_heads, spec.T, spec.d, spec.block, spec.block,
+                         spec.k_top, True, spec.dtype)
+    rng = np.random.default_rng(1234)
+    threads = so.threads()
+
+    def run(n):
+        rows = np.sort(rng.choice(spec.n_rows, size=min(n, spec.n_rows), replace=False))
+        t0 = time.perf_counter()
+        res = so.build_mask_rows(p, w.q, w.k, rows)
+        so.sparse_attention_rows(p, w.q, w.k, w.v, res["mask"], rows)
+        return time.perf_counter() - t0, len(rows)
+
+    t_probe, n_probe = run(2 * threads)
+    n = int(max(2 * threads, min(spec.n_rows, seconds / max(t_probe, 1e-6) * n_probe)))
+    t, n = run(n)
+    return n * spec.block / t, threads, f"{n} seeded rows of {spec.n_rows} (mask + attention), {t:.1f} s wall"
+
+
+def run_reference(args):
+    """The oracle as the reference arm: each step is a bounded row sample of the same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy as np
+
+    from oracle import stream_oracle as so
+    from paper_2510_19875_b200 import workloads as wl
+
+    spec = get_spec(args)
+    w = wl.generate(spec)
+    p = so.OracleProblem(spec.batch, spec.n_q_heads, spec.n_kv_heads, spec.T, spec.d, spec.block, spec.block,
+                         spec.k_top, True, spec.dtype)
+    threads = so.threads()
+    rng = np.random.default_rng(1234)
+    budget = 120.0 / max(1, args.steps + args.warmup)  # whole run within a few minutes
+
+    def step(n):
+        rows = np.sort(rng.choice(spec.n_rows, size=min(n, spec.n_rows), replace=False))
+        t0 = time.perf_counter()
+        res = so.build_mask_rows(p, w.q, w.k, rows)
+        so.sparse_attention_rows(p, w.q, w.k, w.v, res["mask"], rows)
+        return time.perf_counter() - t0
+
+    t_probe = step(2 * threads)
+    n = int(max(2 * threads, min(spec.n_rows, budget / max(t_probe, 1e-6) * 2 * threads)))
+    for _ in range(args.warmup):
+        step(n)
+    times = [step(n) for _ in range(args.steps)]
+    total = sum(times)
+    value = n * spec.block * args.steps / total
+    sample = f"{n} seeded rows of {spec.n_rows} per step (mask + attention)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": workload_config(spec, {"sample": sample}),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2510_19875_b200 import stream as S
+    from paper_2510_19875_b200 import workloads as wl
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path for the library")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    spec = get_spec(args, rank)
+    w = wl.generate(spec)
+    qh, kh, vh = w.torch_tensors("cpu")
+    q, k, v = qh.to(dev), kh.to(dev), vh.to(dev)
+    kw = dict(block_q=spec.block, block_k=spec.block, k_top=spec.k_top)
+    p = S.make_problem(q, k, impl=args.kernels, **kw)
+    nqb = S.n_query_blocks(p)
+    mask = torch.empty((spec.batch, spec.n_q_heads, nqb, spec.k_top), dtype=torch.int32, device=dev)
+    out = torch.empty_like(q)
+    ws = S.new_workspace(p, dev)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        S.stream_build_mask(p, q, k, mask, None, ws, ws.numel(), stream)
+        S.stream_sparse_attention(p, q, k, v, mask, 0.0, out, stream)
+
+    for _ in range(args.warmup):
+        step()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t_begin.record()
+    for i in range(args.steps):
+        ev[i][0].record()
+        S.stream_build_mask(p, q, k, mask, None, ws, ws.numel(), stream)
+        ev[i][1].record()
+        S.stream_sparse_attention(p, q, k, v, mask, 0.0, out, stream)
+        ev[i][2].record()
+    t_end.record()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = t_begin.elapsed_time(t_end)
+    mask_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in ev)
+    attn_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in ev)
+    stats = S.stream_read_stats(ws, stream)
+    kept = int((mask >= 0).sum().item())
+
+    # end to end through the host entry point: pinned host tensors in, mask + output back
+    e2e = None
+    if not args.no_e2e:
+        qp, kp, vp = qh.pin_memory(), kh.pin_memory(), vh.pin_memory()
+        mask_host = torch.empty(mask.shape, dtype=torch.int32).pin_memory()
+        out_host = torch.empty(out.shape, dtype=out.dtype).pin_memory()
+        del out
+        ph = S.make_problem(qp, kp, impl=args.kernels, **kw)
+        staging = torch.empty(S.stream_host_staging_bytes(ph), dtype=torch.uint8, device=dev)
+        n_e2e = max(1, min(args.steps, 5))
+        for _ in range(2):
+            S.stream_run_host(ph, qp, kp, vp, mask_host, out_host, 0.0, staging, staging.numel(), stream)
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(n_e2e):
+            S.stream_run_host(ph, qp, kp, vp, mask_host, out_host, 0.0, staging, staging.numel(), stream)
+        b.record()
+        torch.cuda.synchronize()
+        e2e_ms = a.elapsed_time(b) / n_e2e
+        assert torch.equal(mask_host, mask.cpu()), "host path produced a different mask"
+        e2e = {"ms": e2e_ms, "steps": n_e2e,
+               "h2d": qp.numel() * qp.element_size() + 2 * kp.numel() * kp.element_size(),
+               "d2h": mask_host.numel() * 4 + out_host.numel() * out_host.element_size()}
+
+    times = torch.tensor([total_ms, mask_ms, attn_ms, e2e["ms"] if e2e else 0.0], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    total_ms, mask_ms, attn_ms, e2e_ms = times.tolist()
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    units = spec.batch * spec.n_q_heads * spec.T  # query-token-heads per rank per step
+    esz = 2 if spec.dtype == "bf16" else 4
+    S_tiles = int(stats.tiles_scored)
+    alg_bytes = S_tiles * spec.block * spec.d * esz + units * spec.d * esz + spec.n_rows * spec.k_top * 4
+    peak, peak_kind = hbm_peak()
+    achieved = alg_bytes / (mask_ms * 1e-3) / 1e9
+    traffic = ncu_traffic("stream_build_mask", units)
+    attn_bytes = kept * 2 * spec.block * spec.d * esz + 2 * units * spec.d * esz
+    line = {
+        "metric": METRIC, "value": world * units * args.steps / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": spec.dtype, "data": "synthetic",
+        "config": workload_config(spec, {"l2": "inputs larger than L2 (Q+K+V %.0f MiB per step)" % (
+            (q.numel() + 2 * k.numel()) * esz / 2**20), "kernels": args.kernels, "per_rank": "one independent layer each"}),
+        "mask_build": {"ms": mask_ms, "value": units / (mask_ms * 1e-3), "unit": UNIT, "tiles_scored": S_tiles,
+                       "tensor_tflops": S_tiles * 2.0 * spec.block * spec.block * spec.d / (mask_ms * 1e-3) / 1e12},
+        "sparse_attention": {"ms": attn_ms, "kept_blocks": kept, "algorithmic_gbs": attn_bytes / (attn_ms * 1e-3) / 1e9},
+        "roofline": {"kernel": "stream_build_mask", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "traffic": traffic, "peak_kind": f"of {peak_kind}",
+                     "algorithmic_bytes": alg_bytes, "frac_of_8TBs_nominal": achieved / 8000.0},
+        "clocks": clocks,
+        "gpu_launches": 2 * args.steps,
+    }
+    if e2e:
+        line["e2e"] = {"value": world * units / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+                       "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"], "steps": e2e["steps"]}
+    if not args.no_cpu_baseline:
+        del q, k, v
+        rate, threads, sample = oracle_sample_rate(spec, w, args.cpu_seconds)
+        line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

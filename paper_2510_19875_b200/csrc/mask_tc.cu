@@ -1,10 +1,574 @@
-// Tensor-core (tcgen05) Stream mask kernel. Placeholder until the kernel lands.
+// Tensor-core Stream mask kernel for sm_100a: bf16, d = 128, 64 x 64 blocks, k_top <= 32.
+//
+// One persistent CTA per SM works through "groups": up to four query heads of one kv head at
+// one query block. Their Q tiles stay in shared memory for the whole hierarchy (Algorithm 2).
+// Candidate key blocks are fetched by TMA (128-byte swizzle) two at a time into a ring of
+// stages; one tcgen05.mma chain per (stage, row) computes K_pair (128 x 128) x Q_row^T (128 x 64)
+// into a 64-column TMEM slot; four epilogue warps reduce the slot to the two masked tile maxima
+// (Eq. 4 under C); a controller warp keeps each row's nodes in registers, ranks the 2k branch
+// scores (higher score, then lower block index), compacts the survivors with ballots and
+// publishes the next level's fetch list. The first level's representatives are the same for
+// every row of a group, so one fetched stage serves all its rows; from the second level on a
+// left branch inherits its parent's score and only right branches are fetched.
+//
+// Roles (256 threads): warp 0 TMA producer, warp 1 MMA issuer + TMEM owner, warp 2 controller,
+// warps 4..7 epilogue (TMEM lane quarter = warp % 4). All roles walk the same fixed unit order
+// (level 1: stage-major, row-minor; later levels: row-major), synchronised by mbarriers only.
+// Every wait is bounded: on a timeout the CTA records an error code in the workspace header,
+// raises a shared abort flag, drains its own copies and leaves.
+#include <cuda.h>
+#include <math_constants.h>
+
 #include "common.cuh"
 
 namespace stream {
-bool mask_tc_supported(const Geom &, int) { return false; }
-stream_status launch_mask_tc(const Geom &, const void *, const void *, int32_t *, float *, WorkspaceHeader *, cudaStream_t) {
-    set_error("tensor-core mask kernel not built");
-    return STREAM_ERR_UNSUPPORTED;
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kR = 4;          // rows (query heads) per group
+constexpr int kStages = 4;     // K-pair stages
+constexpr int kSlots = 8;      // TMEM accumulator slots of 64 fp32 columns
+constexpr int kBlk = 64, kD = 128;
+constexpr int kHalfTile = kBlk * 128;          // 64 rows x 128 bytes (one 64-channel half)
+constexpr int kStageBytes = 4 * kHalfTile;     // [2 channel halves][2 tiles]
+constexpr int kQBytes = 2 * kR * kHalfTile;    // [2 channel halves][kR rows]
+constexpr int kMaxJobs = 64;
+constexpr long long kWaitCycles = 1ll << 31;   // ~1 s: far beyond any legitimate wait
+
+struct Tail {
+    unsigned long long full[kStages], empty[kStages], tmem_full[kSlots], tmem_empty[kSlots];
+    unsigned long long q_full, jobs_ready[kR + 1], scores_done[kR];
+    unsigned int tmem_base;
+    int abort_flag;
+    int grp_id, grp_b, grp_kvh, grp_qb, grp_h0, grp_R;
+    int n_jobs[kR + 1];
+    int jobs_blk[kR + 1][kMaxJobs];
+    float part[kR][kMaxJobs][2];
+    int node_f[32], node_l[32];
+    float node_s[32];
+};
+constexpr int kSmemBytes = kQBytes + kStages * kStageBytes + (int)sizeof(Tail) + 1024;
+
+// ----------------------------------------------------------------------------------------------
+// PTX wrappers
+// ----------------------------------------------------------------------------------------------
+__device__ __forceinline__ unsigned smem_u32(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
+__device__ __forceinline__ void mbar_arrive(unsigned bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(unsigned bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
+    unsigned ok;
+    asm volatile(
+        "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// Bounded wait. Returns false if the CTA is aborting (or this wait ran out, which starts an abort).
+__device__ __noinline__ bool mbar_wait(unsigned bar, unsigned parity, Tail *tl, WorkspaceHeader *ws, unsigned code) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*(volatile int *)&tl->abort_flag) return false;
+        if (clock64() - t0 > kWaitCycles) {
+            *(volatile int *)&tl->abort_flag = 1;
+            if (atomicCAS(&ws->error, 0u, code) == 0u) ws->error_info = blockIdx.x;
+            return false;
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_4d(unsigned dst, const CUtensorMap *map, unsigned bar, int c0, int c1, int c2,
+                                            int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"((unsigned long long)map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(unsigned bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tc_mma_bf16(unsigned d_tmem, unsigned long long adesc, unsigned long long bdesc,
+                                            unsigned idesc, unsigned accumulate) {
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// 32 lanes x 32 consecutive fp32 columns of TMEM: thread i gets lane (base lane + i).
+__device__ __forceinline__ void tmem_ld_32x32(unsigned taddr, float *v) {
+    unsigned r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+__device__ __forceinline__ float warp_max(float x) {
+    float r;
+    asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(x));
+    return r;
+}
+
+// Shared-memory matrix descriptor: K-major rows of 128 bytes, 128-byte swizzle, 8-row groups
+// 1024 bytes apart, descriptor version 1 (sm_100).
+__device__ __forceinline__ unsigned long long smem_desc(unsigned addr) {
+    return (unsigned long long)((addr >> 4) & 0x3FFF) | (1ull << 16) | ((unsigned long long)(1024 >> 4) << 32) |
+           (1ull << 46) | (2ull << 61);
+}
+
+// kind::f16 instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = 64.
+constexpr unsigned kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
+
+struct Params {
+    Geom g;
+    int n_groups, n_chunks;
+    int32_t *mask;
+    float *score;
+    WorkspaceHeader *ws;
+};
+
+// ----------------------------------------------------------------------------------------------
+// Roles
+// ----------------------------------------------------------------------------------------------
+struct Ring {  // position in a ring of barriers with phase tracking
+    int idx = 0;
+    unsigned phase = 0;
+    __device__ void advance(int n) {
+        if (++idx == n) { idx = 0; phase ^= 1; }
+    }
+};
+
+__device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUtensorMap *tk, Tail *tl, unsigned q_smem,
+                              unsigned k_smem) {
+    const Geom &g = P.g;
+    Ring st;
+    unsigned grp_par = 0, jr_par[kR] = {0, 0, 0, 0};
+    for (;;) {
+        if (!mbar_wait(smem_u32(&tl->jobs_ready[kR]), grp_par, tl, P.ws, 101)) return;
+        grp_par ^= 1;
+        if (tl->grp_id < 0) return;
+        const int b = tl->grp_b, kvh = tl->grp_kvh, qb = tl->grp_qb, h0 = tl->grp_h0, R = tl->grp_R;
+        // Q tiles of the group's rows (previous group's MMAs are all complete by now)
+        mbar_arrive_expect_tx(smem_u32(&tl->q_full), (unsigned)(R * 2 * kHalfTile));
+        for (int r = 0; r < R; ++r)
+            for (int c = 0; c < 2; ++c)
+                tma_load_4d(q_smem + (c * kR + r) * kHalfTile, tq, smem_u32(&tl->q_full), c * 64, qb * kBlk, h0 + r, b);
+        for (int level = 0; level < g.levels; ++level) {
+            const int lists = level == 0 ? 1 : R;
+            for (int x = 0; x < lists; ++x) {
+                const int li = level == 0 ? kR : x;
+                if (level > 0) {
+                    if (!mbar_wait(smem_u32(&tl->jobs_ready[x]), jr_par[x], tl, P.ws, 102)) return;
+                    jr_par[x] ^= 1;
+                }
+                const int n = tl->n_jobs[li];
+                for (int j = 0; j < n; j += 2) {
+                    if (!mbar_wait(smem_u32(&tl->empty[st.idx]), st.phase ^ 1, tl, P.ws, 103)) return;
+                    const int two = (j + 1 < n);
+                    const unsigned bar = smem_u32(&tl->full[st.idx]);
+                    const unsigned dst = k_smem + st.idx * kStageBytes;
+                    mbar_arrive_expect_tx(bar, (unsigned)((two ? 4 : 2) * kHalfTile));
+                    for (int t = 0; t <= two; ++t) {
+                        const int blk = tl->jobs_blk[li][j + t];
+                        for (int c = 0; c < 2; ++c)
+                            tma_load_4d(dst + (c * 2 + t) * kHalfTile, tk, bar, c * 64, blk * kBlk, kvh, b);
+                    }
+                    st.advance(kStages);
+                }
+            }
+        }
+    }
+}
+
+__device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_smem, unsigned tmem_base) {
+    const Geom &g = P.g;
+    Ring st, sl;
+    unsigned grp_par = 0, q_par = 0, jr_par[kR] = {0, 0, 0, 0};
+    for (;;) {
+        if (!mbar_wait(smem_u32(&tl->jobs_ready[kR]), grp_par, tl, P.ws, 201)) return;
+        grp_par ^= 1;
+        if (tl->grp_id < 0) return;
+        const int R = tl->grp_R;
+        if (!mbar_wait(smem_u32(&tl->q_full), q_par, tl, P.ws, 202)) return;
+        q_par ^= 1;
+        for (int level = 0; level < g.levels; ++level) {
+            const int lists = level == 0 ? 1 : R;
+            for (int x = 0; x < lists; ++x) {
+                const int li = level == 0 ? kR : x;
+                if (level > 0) {
+                    if (!mbar_wait(smem_u32(&tl->jobs_ready[x]), jr_par[x], tl, P.ws, 203)) return;
+                    jr_par[x] ^= 1;
+                }
+                const int n = tl->n_jobs[li];
+                for (int j = 0; j < n; j += 2) {
+                    if (!mbar_wait(smem_u32(&tl->full[st.idx]), st.phase, tl, P.ws, 204)) return;
+                    const unsigned a_base = k_smem + st.idx * kStageBytes;
+                    const int r0 = level == 0 ? 0 : x, r1 = level == 0 ? R : x + 1;
+                    for (int r = r0; r < r1; ++r) {
+                        if (!mbar_wait(smem_u32(&tl->tmem_empty[sl.idx]), sl.phase ^ 1, tl, P.ws, 205)) return;
+                        tc_fence_after();
+                        const unsigned d_tmem = tmem_base + sl.idx * 64;
+#pragma unroll
+                        for (int c = 0; c < 2; ++c)
+#pragma unroll
+                            for (int k4 = 0; k4 < 4; ++k4)
+                                tc_mma_bf16(d_tmem, smem_desc(a_base + c * 2 * kHalfTile + k4 * 32),
+                                            smem_desc(q_smem + (c * kR + r) * kHalfTile + k4 * 32), kIdesc, (c | k4) != 0);
+                        tc_commit(smem_u32(&tl->tmem_full[sl.idx]));
+                        sl.advance(kSlots);
+                    }
+                    tc_commit(smem_u32(&tl->empty[st.idx]));
+                    st.advance(kStages);
+                }
+            }
+        }
+    }
+}
+
+__device__ void epilogue_role(const Params &P, Tail *tl, unsigned tmem_base, int wq, int lane) {
+    const Geom &g = P.g;
+    Ring sl;
+    unsigned grp_par = 0, jr_par[kR] = {0, 0, 0, 0};
+    const int tile = wq >> 1;                // which tile of the pair this warp's lanes hold
+    const int key = (wq & 1) * 32 + lane;    // key index inside the tile
+    for (;;) {
+        if (!mbar_wait(smem_u32(&tl->jobs_ready[kR]), grp_par, tl, P.ws, 301)) return;
+        grp_par ^= 1;
+        if (tl->grp_id < 0) return;
+        const int R = tl->grp_R, qb = tl->grp_qb;
+        const long long rem_q = g.T - (long long)qb * kBlk;
+        const int m_lim = rem_q < kBlk ? (int)rem_q : kBlk;  // query tokens of this block inside T
+        for (int level = 0; level < g.levels; ++level) {
+            const int lists = level == 0 ? 1 : R;
+            for (int x = 0; x < lists; ++x) {
+                const int li = level == 0 ? kR : x;
+                if (level > 0) {
+                    if (!mbar_wait(smem_u32(&tl->jobs_ready[x]), jr_par[x], tl, P.ws, 302)) return;
+                    jr_par[x] ^= 1;
+                }
+                const int n = tl->n_jobs[li];
+                for (int j = 0; j < n; j += 2) {
+                    const int c = j + tile;
+                    const int blk = c < n ? tl->jobs_blk[li][c] : -1;
+                    const int r0 = level == 0 ? 0 : x, r1 = level == 0 ? R : x + 1;
+                    for (int r = r0; r < r1; ++r) {
+                        if (!mbar_wait(smem_u32(&tl->tmem_full[sl.idx]), sl.phase, tl, P.ws, 303)) return;
+                        tc_fence_after();
+                        if (blk >= 0) {
+                            const unsigned taddr = tmem_base + sl.idx * 64 + ((unsigned)(wq * 32) << 16);
+                            float v[64];
+                            tmem_ld_32x32(taddr, v);
+                            tmem_ld_32x32(taddr + 32, v + 32);
+                            // allowed queries for this key: inside T, and not before the key if causal
+                            const long long rem_k = g.T - (long long)blk * kBlk;
+                            int lo = (g.causal && blk == qb) ? key : 0;
+                            if (key >= rem_k) lo = kBlk;  // key beyond T
+                            float best = -CUDART_INF_F;
+                            if (lo == 0 && m_lim == kBlk) {
+#pragma unroll
+                                for (int i = 0; i < 64; ++i) best = fmaxf(best, v[i]);
+                            } else {
+#pragma unroll
+                                for (int i = 0; i < 64; ++i)
+                                    if (i >= lo && i < m_lim) best = fmaxf(best, v[i]);
+                            }
+                            best = warp_max(best);
+                            if (lane == 0) tl->part[r][c][wq & 1] = best;
+                        }
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&tl->tmem_empty[sl.idx]));
+                        sl.advance(kSlots);
+                    }
+                }
+                // this list is done for rows r0..r1: tell the controller
+                if (lane == 0) {
+                    const int r0 = level == 0 ? 0 : x, r1 = level == 0 ? R : x + 1;
+                    for (int r = r0; r < r1; ++r) mbar_arrive(smem_u32(&tl->scores_done[r]));
+                }
+            }
+        }
+    }
+}
+
+// Controller helpers -----------------------------------------------------------------------------
+struct Keep { bool l, r; };
+
+// Rank the (up to) 64 candidates held two per lane; keep the k best by (score desc, index asc).
+__device__ __forceinline__ Keep select_topk(bool vl, float sl, bool vr, float sr, int k, int lane) {
+    const int total = __popc(__ballot_sync(0xffffffffu, vl)) + __popc(__ballot_sync(0xffffffffu, vr));
+    if (total <= k) return {vl, vr};
+    const float el = vl ? sl : -CUDART_INF_F, er = vr ? sr : -CUDART_INF_F;
+    int rank_l = 0, rank_r = 0;
+#pragma unroll 8
+    for (int j = 0; j < 32; ++j) {
+        const float ol = __shfl_sync(0xffffffffu, el, j), orr = __shfl_sync(0xffffffffu, er, j);
+        rank_l += (ol > el) || (ol == el && j < lane);
+        rank_l += (orr > el) || (orr == el && j < lane);
+        rank_r += (ol > er) || (ol == er && j <= lane);
+        rank_r += (orr > er) || (orr == er && j < lane);
+    }
+    return {vl && rank_l < k, vr && rank_r < k};
+}
+
+__device__ void controller_role(const Params &P, Tail *tl, int lane) {
+    const Geom &g = P.g;
+    const unsigned lt = (1u << lane) - 1u;
+    unsigned sd_par[kR] = {0, 0, 0, 0};
+    for (;;) {
+        int id = 0;
+        if (lane == 0) id = (int)atomicAdd(&P.ws->work_counter, 1u);
+        id = __shfl_sync(0xffffffffu, id, 0);
+        const bool done = id >= P.n_groups || *(volatile int *)&tl->abort_flag;
+        int b = 0, kvh = 0, qb = 0, h0 = 0, R = 0;
+        if (!done) {
+            const int per = g.n_qb * P.n_chunks;
+            const int bkv = id / per, rem = id % per;
+            b = bkv / g.G; kvh = bkv % g.G;
+            qb = g.n_qb - 1 - rem / P.n_chunks;  // late (expensive) query blocks first
+            const int chunk = rem % P.n_chunks;
+            h0 = kvh * g.hpg + chunk * kR;
+            R = min(kR, g.hpg - chunk * kR);
+        }
+        const int q_lim = last_valid_block(g, qb);
+        // initial nodes: lane i holds node i (the same for every row of the group)
+        int f0 = (int)(((long long)lane * g.N_k) / g.k_top), l0 = (int)(((long long)(lane + 1) * g.N_k) / g.k_top) - 1;
+        const bool v0 = !done && lane < g.k_top && f0 <= l0 && f0 <= q_lim;
+        const int m0 = (f0 + l0) / 2;
+        const bool vl1 = v0, vr1 = v0 && m0 + 1 <= l0 && m0 + 1 <= q_lim;
+        const unsigned bl = __ballot_sync(0xffffffffu, vl1), br = __ballot_sync(0xffffffffu, vr1);
+        const int c_l1 = __popc(bl & lt) + __popc(br & lt), c_r1 = c_l1 + (vl1 ? 1 : 0);
+        if (vl1) tl->jobs_blk[kR][c_l1] = f0;
+        if (vr1) tl->jobs_blk[kR][c_r1] = m0 + 1;
+        const int n1 = __popc(bl) + __popc(br);
+        if (lane == 0) {
+            tl->n_jobs[kR] = n1;
+            tl->grp_id = done ? -1 : id; tl->grp_b = b; tl->grp_kvh = kvh; tl->grp_qb = qb; tl->grp_h0 = h0; tl->grp_R = R;
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&tl->jobs_ready[kR]));
+        if (done) return;
+
+        int nf[kR], nl[kR], my_c[kR], n_nodes[kR];
+        float ns[kR];
+        bool has_r[kR];
+        unsigned tiles = (unsigned)(n1 * R);
+        for (int level = 0; level < g.levels; ++level) {
+#pragma unroll
+            for (int r = 0; r < kR; ++r) {
+                if (r >= R) continue;
+                if (!mbar_wait(smem_u32(&tl->scores_done[r]), sd_par[r], tl, P.ws, 401)) return;
+                sd_par[r] ^= 1;
+                // candidates of this lane's node: left (f : m) and right (m + 1 : l)
+                int f, l, m;
+                bool vl, vr;
+                float sl, sr = -CUDART_INF_F;
+                if (level == 0) {
+                    f = f0; l = l0; m = m0; vl = vl1; vr = vr1;
+                    sl = vl ? fmaxf(tl->part[r][c_l1][0], tl->part[r][c_l1][1]) : -CUDART_INF_F;
+                    if (vr) sr = fmaxf(tl->part[r][c_r1][0], tl->part[r][c_r1][1]);
+                } else {
+                    f = nf[r]; l = nl[r]; m = (f + l) / 2;
+                    vl = lane < n_nodes[r]; vr = has_r[r];
+                    sl = ns[r];
+                    if (vr) sr = fmaxf(tl->part[r][my_c[r]][0], tl->part[r][my_c[r]][1]);
+                }
+                const Keep kp = select_topk(vl, sl, vr, sr, g.k_top, lane);
+                const unsigned kl = __ballot_sync(0xffffffffu, kp.l), kr = __ballot_sync(0xffffffffu, kp.r);
+                const int pos_l = __popc(kl & lt) + __popc(kr & lt), pos_r = pos_l + (kp.l ? 1 : 0);
+                __syncwarp();
+                if (kp.l) { tl->node_f[pos_l] = f; tl->node_l[pos_l] = m; tl->node_s[pos_l] = sl; }
+                if (kp.r) { tl->node_f[pos_r] = m + 1; tl->node_l[pos_r] = l; tl->node_s[pos_r] = sr; }
+                __syncwarp();
+                n_nodes[r] = __popc(kl) + __popc(kr);
+                const bool live = lane < n_nodes[r];
+                nf[r] = live ? tl->node_f[lane] : 0;
+                nl[r] = live ? tl->node_l[lane] : -1;
+                ns[r] = live ? tl->node_s[lane] : -CUDART_INF_F;
+                if (level + 1 < g.levels) {
+                    // next level: only right branches need a tile; left ones keep the node's score
+                    const int mm = (nf[r] + nl[r]) / 2;
+                    has_r[r] = live && nl[r] > nf[r] && mm + 1 <= q_lim;
+                    const unsigned hb = __ballot_sync(0xffffffffu, has_r[r]);
+                    my_c[r] = __popc(hb & lt);
+                    if (has_r[r]) tl->jobs_blk[r][my_c[r]] = mm + 1;
+                    if (lane == 0) tl->n_jobs[r] = __popc(hb);
+                    tiles += (unsigned)__popc(hb);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&tl->jobs_ready[r]));
+                } else {
+                    // emit I[q, :]: first block of every surviving node, ascending, -1 padded
+                    const long long row = ((long long)b * g.H + (h0 + r)) * g.n_qb + qb;
+                    if (lane < g.k_top) {
+                        P.mask[row * g.k_top + lane] = live ? nf[r] : -1;
+                        if (P.score != nullptr) P.score[row * g.k_top + lane] = live ? ns[r] : -CUDART_INF_F;
+                    }
+                }
+            }
+        }
+        if (lane == 0) {
+            atomicAdd(&P.ws->tiles_scored, (unsigned long long)tiles);
+            atomicAdd(&P.ws->rows, (unsigned long long)R);
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+mask_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k, Params P) {
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    unsigned char *smem = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const unsigned q_smem = smem_u32(smem), k_smem = q_smem + kQBytes;
+    Tail *tl = (Tail *)(smem + kQBytes + kStages * kStageBytes);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kStages; ++i) { mbar_init(smem_u32(&tl->full[i]), 1); mbar_init(smem_u32(&tl->empty[i]), 1); }
+        for (int i = 0; i < kSlots; ++i) { mbar_init(smem_u32(&tl->tmem_full[i]), 1); mbar_init(smem_u32(&tl->tmem_empty[i]), 4); }
+        mbar_init(smem_u32(&tl->q_full), 1);
+        for (int i = 0; i <= kR; ++i) mbar_init(smem_u32(&tl->jobs_ready[i]), 1);
+        for (int i = 0; i < kR; ++i) mbar_init(smem_u32(&tl->scores_done[i]), 4);
+        tl->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {  // TMEM: all 512 columns (one CTA per SM)
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tl->tmem_base)), "r"(512)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const unsigned tmem_base = tl->tmem_base;
+
+    if (warp == 0) {
+        if (lane == 0) producer_role(P, &tmap_q, &tmap_k, tl, q_smem, k_smem);
+    } else if (warp == 1) {
+        if (lane == 0) mma_role(P, tl, q_smem, k_smem, tmem_base);
+    } else if (warp == 2) {
+        controller_role(P, tl, lane);
+    } else if (warp >= 4) {
+        epilogue_role(P, tl, tmem_base, warp & 3, lane);
+    }
+    __syncwarp();
+
+    // Teardown. After an abort, copies and MMAs may still be in flight: give every stage and slot
+    // barrier a bounded chance to complete before shared memory and TMEM are given back.
+    if (*(volatile int *)&tl->abort_flag) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < (1ll << 22)) { }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+    }
+}
+
+// ----------------------------------------------------------------------------------------------
+// Host side
+// ----------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (fn == nullptr) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// [batch, heads, T, 128] bf16 with element strides -> 4-D map with a 64 x 64 box, 128-byte swizzle.
+stream_status make_map(CUtensorMap *map, const void *base, long long T, int heads, int batch, long long s_t,
+                       long long s_h, long long s_b, const char *what) {
+    EncodeTiledFn fn = encode_fn();
+    if (fn == nullptr) { set_error("cuTensorMapEncodeTiled is not available from this driver"); return STREAM_ERR_CUDA; }
+    // extents of 1 may come with arbitrary strides: give them a well-formed one
+    if (heads == 1) s_h = s_t * T;
+    if (batch == 1) s_b = s_h * heads;
+    cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)T, (cuuint64_t)heads, (cuuint64_t)batch};
+    cuuint64_t strides[3] = {(cuuint64_t)s_t * 2, (cuuint64_t)s_h * 2, (cuuint64_t)s_b * 2};
+    cuuint32_t box[4] = {64, 64, 1, 1}, estr[4] = {1, 1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled(%s) failed with %d", what, (int)r); return STREAM_ERR_CUDA; }
+    return STREAM_OK;
+}
+
+}  // namespace
+
+bool mask_tc_supported(const Geom &g, int dtype) {
+    auto ok_stride = [](long long s) { return s % 8 == 0; };  // 16-byte multiples for TMA
+    return dtype == STREAM_BF16 && g.d == kD && g.bq == kBlk && g.bk == kBlk && g.k_top <= 32 && g.levels >= 1 &&
+           ok_stride(g.qs_t) && ok_stride(g.qs_h) && ok_stride(g.qs_b) && ok_stride(g.ks_t) && ok_stride(g.ks_h) &&
+           ok_stride(g.ks_b);
+}
+
+stream_status launch_mask_tc(const Geom &g, const void *q, const void *k, int32_t *mask, float *score,
+                             WorkspaceHeader *ws, cudaStream_t st) {
+    if (((uintptr_t)q & 15) != 0 || ((uintptr_t)k & 15) != 0) {
+        set_error("tensor-core mask kernel needs 16-byte aligned q and k");
+        return STREAM_ERR_UNSUPPORTED;
+    }
+    CUtensorMap tq, tk;
+    stream_status rc = make_map(&tq, q, g.T, g.H, g.batch, g.qs_t, g.qs_h, g.qs_b, "q");
+    if (rc != STREAM_OK) return rc;
+    rc = make_map(&tk, k, g.T, g.G, g.batch, g.ks_t, g.ks_h, g.ks_b, "k");
+    if (rc != STREAM_OK) return rc;
+    Params P;
+    P.g = g;
+    P.n_chunks = (g.hpg + kR - 1) / kR;
+    long long n_groups = (long long)g.batch * g.G * g.n_qb * P.n_chunks;
+    P.n_groups = (int)n_groups;
+    P.mask = mask; P.score = score; P.ws = ws;
+    static int n_sm = 0;
+    if (n_sm == 0) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaError_t e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
+    }
+    cudaError_t e = cudaFuncSetAttribute(mask_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(mask_tc)");
+    int grid = (int)(n_groups < n_sm ? n_groups : n_sm);
+    mask_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(tq, tk, P);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "mask_tc launch");
+    return STREAM_OK;
+}
+
 }  // namespace stream

@@ -83,6 +83,46 @@ def test_mask_generic_small(S, kw):
     assert_mask_parity(S, w, None, impl="generic", score_cache=False)
 
 
+def tc_spec(**kw):
+    base = dict(name="tc", seed=7, batch=1, n_q_heads=4, n_kv_heads=1, T=4096, d=128, block=64, k_top=8, dtype="bf16", sink=True)
+    base.update(kw)
+    return wl.WorkloadSpec(**base)
+
+
+TC_CASES = [
+    dict(),                                                   # one kv head, four rows per group, 3 levels
+    dict(T=2048, k_top=16, n_q_heads=8, n_kv_heads=2),        # N_k = 2k: a single level
+    dict(T=8192, k_top=32, n_q_heads=2, n_kv_heads=2),        # one row per group
+    dict(T=5000, k_top=5, n_q_heads=7, n_kv_heads=1),         # ragged T, odd k, groups of 4 + 3 heads
+    dict(T=3000, k_top=3, n_q_heads=6, n_kv_heads=2, batch=2, local=True),
+    dict(T=16384, k_top=1, n_q_heads=1, n_kv_heads=1),        # k = 1
+    dict(T=1024, k_top=32, n_q_heads=4, n_kv_heads=4),        # k > N_k
+    dict(T=100, k_top=4, n_q_heads=4, n_kv_heads=2),          # two key blocks, ragged
+]
+
+
+@pytest.mark.parametrize("kw", TC_CASES)
+def test_mask_tensor_core_small(S, kw):
+    w = wl.generate(tc_spec(**kw))
+    assert_mask_parity(S, w, None, impl="tensor", score_cache=False)
+
+
+def test_mask_tensor_core_non_causal(S):
+    w = wl.generate(tc_spec(T=3000, k_top=6))
+    assert_mask_parity(S, w, None, impl="tensor", score_cache=False, causal=False)
+
+
+def test_mask_tensor_core_matches_generic_kernel(S):
+    w = wl.generate(tc_spec(T=8192, k_top=16, n_q_heads=8, n_kv_heads=2, anchors=True))
+    a = run_mask(S, w, impl="tensor", want_scores=True)
+    b = run_mask(S, w, impl="generic", want_scores=True)
+    same = (a.mask == b.mask).all(-1)
+    assert same.float().mean().item() > 0.97  # the rest are near-ties resolved by rounding
+    fin = torch.isfinite(b.scores[same])
+    torch.testing.assert_close(a.scores[same][fin], b.scores[same][fin], rtol=2e-5, atol=2e-5)
+    assert a.stats().tiles_scored == b.stats().tiles_scored or not same.all()
+
+
 @pytest.mark.parametrize("bq,bk", [(16, 32), (32, 8), (1, 16), (24, 16)])
 def test_mask_generic_unequal_blocks(S, bq, bk):
     w = wl.generate(small_spec(T=700, k_top=5))

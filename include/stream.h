@@ -108,6 +108,29 @@ stream_status stream_build_mask(const stream_problem *p, const void *q, const vo
                                 float *score_out, void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * stream_build_mask without a caller-provided workspace and without any allocation. (The paper
+ * has no counterpart to this entry point; it exists for deployment.)
+ *
+ * For callers that cannot get device memory when they call: a host application that reserved all
+ * of HBM for its own pool at start-up, or a latency-critical loop that must not hit the implicit
+ * synchronisation of cudaMalloc / cudaFree. The kernel's scratch (work counter and counters, see
+ * stream_stats) lives in a 4096-byte device array built into the library, which each GPU that
+ * loads the library holds until the process exits. Same arguments, results and errors as
+ * stream_build_mask otherwise; a problem whose scratch need exceeded 4096 bytes would be refused
+ * with STREAM_ERR_WORKSPACE (no current problem does). The call allocates and frees nothing.
+ *
+ *   - The first call on each device looks up the array's device address (a one-time host-side
+ *     query, made with that device current). Make that first call outside any stream capture.
+ *   - All calls on a device share the one array and it keeps the previous call's contents; each
+ *     call clears what it needs on `cuda_stream` before its kernel. Two calls that can overlap on
+ *     the GPU (different streams, no dependency) race on it: serialise them, or give the
+ *     overlapping calls stream_build_mask with workspaces of their own.
+ *   - The counters are not readable through this entry point.
+ */
+stream_status stream_build_mask_static(const stream_problem *p, const void *q, const void *k, int32_t *mask_out,
+                                       float *score_out, void *cuda_stream);
+
+/*
  * Block-sparse attention under a Stream mask (Eq. 2 of the paper; the product QK^T * C * M of
  * Figure 1): for every query token, softmax(scale * q.k) over the keys of the row's kept blocks
  * that C allows (element-level causal test inside a block, keys beyond T excluded), times V.

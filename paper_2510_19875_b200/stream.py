@@ -74,6 +74,8 @@ def _load():
     lib.stream_workspace_bytes.argtypes = [P]
     lib.stream_build_mask.restype = ctypes.c_int
     lib.stream_build_mask.argtypes = [P, vp, vp, vp, vp, vp, sz, vp]
+    lib.stream_build_mask_static.restype = ctypes.c_int
+    lib.stream_build_mask_static.argtypes = [P, vp, vp, vp, vp, vp]
     lib.stream_sparse_attention.restype = ctypes.c_int
     lib.stream_sparse_attention.argtypes = [P, vp, vp, vp, vp, ctypes.c_float, vp, vp]
     lib.stream_read_stats.restype = ctypes.c_int
@@ -123,6 +125,12 @@ def stream_workspace_bytes(p: StreamProblem) -> int:
 def stream_build_mask(p: StreamProblem, q, k, mask_out, score_out, workspace, workspace_bytes: int, stream=None) -> None:
     _raise(_load().stream_build_mask(ctypes.byref(p), _addr(q), _addr(k), _addr(mask_out), _addr(score_out),
                                      _addr(workspace), workspace_bytes, _stream_handle(stream)))
+
+
+def stream_build_mask_static(p: StreamProblem, q, k, mask_out, score_out, stream=None) -> None:
+    """Mask build on the library's built-in scratch: no workspace argument, nothing allocated."""
+    _raise(_load().stream_build_mask_static(ctypes.byref(p), _addr(q), _addr(k), _addr(mask_out), _addr(score_out),
+                                            _stream_handle(stream)))
 
 
 def stream_sparse_attention(p: StreamProblem, q, k, v, mask, scale: float, out, stream=None) -> None:

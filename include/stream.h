@@ -44,8 +44,9 @@ typedef enum { STREAM_F32 = 0, STREAM_BF16 = 1 } stream_dtype;
 typedef enum {
     STREAM_IMPL_AUTO = 0,    /* tensor-core kernels when the shape allows, else the generic ones */
     STREAM_IMPL_GENERIC = 1, /* fp32-FMA kernels: any dtype, d in {16,32,64,128}, blocks 1..64 */
-    STREAM_IMPL_TENSOR = 2   /* tcgen05 kernels only: bf16, d = 128, block_q = block_k = 64,
-                                k_top <= 64, causal; otherwise STREAM_ERR_UNSUPPORTED */
+    STREAM_IMPL_TENSOR = 2   /* tcgen05 kernels only: bf16, d = 128, block_q = block_k = 64, strides
+                                that are multiples of 8 elements, 16-byte aligned pointers (and
+                                k_top <= 32 for the mask build); otherwise STREAM_ERR_UNSUPPORTED */
 } stream_impl;
 
 typedef struct {
@@ -152,6 +153,14 @@ stream_status stream_sparse_attention(const stream_problem *p, const void *q, co
  * returns STREAM_ERR_DEVICE_CHECK if the kernel recorded a bounded wait that ran out.
  */
 stream_status stream_read_stats(const void *workspace, stream_stats *out, void *cuda_stream);
+
+/*
+ * Synchronous health check of the kernels that have no workspace to report into (the tensor-core
+ * attention kernel). Waits for `cuda_stream` to drain and returns STREAM_ERR_DEVICE_CHECK if, on
+ * the current device and since the library was loaded, such a kernel gave up on one of its
+ * bounded waits and left early (its output is then incomplete); STREAM_OK otherwise.
+ */
+stream_status stream_check_device_status(void *cuda_stream);
 
 /*
  * Bytes of device staging stream_run_host needs: room for Q, K, V, the mask, the output and the

@@ -144,7 +144,7 @@ stream_status stream_sparse_attention(const stream_problem *p, const void *q, co
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const bool tc_ok = attn_tc_supported(g, p->dtype);
     if (p->impl == STREAM_IMPL_TENSOR && !tc_ok) {
-        set_error("tensor-core attention kernel needs bf16, d = 128, block_q = block_k = 64");
+        set_error("tensor-core attention kernel needs bf16, d = 128, block_q = block_k = 64, 16-byte aligned strides");
         return STREAM_ERR_UNSUPPORTED;
     }
     if (tc_ok && p->impl != STREAM_IMPL_GENERIC) return launch_attn_tc(g, q, k, v, mask, scale, out, st);
@@ -160,6 +160,17 @@ stream_status stream_read_stats(const void *workspace, stream_stats *out, void *
     if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
     if (out->error != 0) {
         set_error("kernel gave up on a bounded wait: code %u, info %u", out->error, out->error_info);
+        return STREAM_ERR_DEVICE_CHECK;
+    }
+    return STREAM_OK;
+}
+
+stream_status stream_check_device_status(void *cuda_stream) {
+    unsigned int words[2] = {0, 0};
+    stream_status rc = read_attn_status(words, (cudaStream_t)cuda_stream);
+    if (rc != STREAM_OK) return rc;
+    if (words[0] != 0) {
+        set_error("attention kernel gave up on a bounded wait: code %u, block %u", words[0], words[1]);
         return STREAM_ERR_DEVICE_CHECK;
     }
     return STREAM_OK;

@@ -1,10 +1,450 @@
-// Tensor-core block-sparse attention kernel. Placeholder until the kernel lands.
-#include "common.cuh"
+// Tensor-core block-sparse attention for sm_100a (Eq. 2 on a Stream mask): bf16, d = 128,
+// 64 x 64 blocks.
+//
+// One persistent CTA per SM works through "pairs": two query heads of one kv head at one query
+// block. Their Q tiles are stacked into one 128-row A operand. For every mask entry e the two
+// rows name one key block each (K_a, K_b, usually different); their tiles are fetched by TMA
+// (128-byte swizzle) and stacked too, so that
+//     S = [Q_0; Q_1] [K_a; K_b]^T      (128 x 128, fp32 in TMEM)
+// holds row 0's logits in its upper-left quadrant and row 1's in its lower-right one. The four
+// softmax warps own one TMEM lane (= one query token) per thread: they read their 64 logits,
+// apply the element-level mask C, update the running maximum and sum (online softmax, fp32), and
+// write P = exp(.) as bf16 into a block-diagonal 128 x 128 A operand in shared memory whose
+// off-diagonal quadrants stay zero. Then
+//     O_e = P [V_a; V_b]               (128 x 128, fp32 in TMEM, V tiles MN-major)
+// gives both rows' contributions in one chain, which the same threads fold into their fp32
+// output registers (o = o * alpha + O_e) one iteration later, so that the tensor core works on
+// the next logits meanwhile.
+//
+// Roles (256 threads): warp 0 TMA producer, warp 1 MMA issuer + TMEM owner, warps 4..7 softmax.
+// Every role derives the same sequence of (pair, entry) from blockIdx and the mask itself; they
+// meet only on mbarriers. Every wait is bounded: on a timeout the CTA records a code in a device
+// status word, raises a shared abort flag, lets its copies drain and leaves.
+#include <math_constants.h>
+
+#include "tc_common.cuh"
 
 namespace stream {
-bool attn_tc_supported(const Geom &, int) { return false; }
-stream_status launch_attn_tc(const Geom &, const void *, const void *, const void *, const int32_t *, float, void *, cudaStream_t) {
-    set_error("tensor-core attention kernel not built");
-    return STREAM_ERR_UNSUPPORTED;
+
+// Status word of the tensor-core attention kernel: 0, or the code of the bounded wait that ran
+// out (with the block index beside it). Read by stream_check_device_status.
+__device__ unsigned int g_attn_status[2];
+
+namespace {
+
+using namespace tc;
+
+constexpr int kThreads = 256;
+constexpr int kBlk = 64, kD = 128;
+constexpr int kHalfTile = kBlk * 128;       // 64 rows x 128 bytes
+constexpr int kOperand = 4 * kHalfTile;     // 128 rows x 256 bytes as [2 column halves][128 rows][128 B]
+constexpr int kKStages = 3, kVStages = 2;
+
+struct Tail {
+    unsigned long long q_full, q_empty;
+    unsigned long long k_full[kKStages], k_empty[kKStages], v_full[kVStages], v_empty[kVStages];
+    unsigned long long s_full[2], s_empty[2], o_full[2], o_empty[2], p_full;
+    unsigned int tmem_base;
+    int abort_flag;
+};
+constexpr int kSmemBytes = (2 + kKStages + kVStages) * kOperand + (int)sizeof(Tail) + 1024;
+static_assert(kSmemBytes <= 232448, "exceeds the shared memory of one CTA");
+
+constexpr unsigned kIdescQK = idesc_bf16(128, 128, false);  // B = stacked K tiles, K-major
+constexpr unsigned kIdescPV = idesc_bf16(128, 128, true);   // B = stacked V tiles, MN-major
+
+struct Params {
+    Geom g;
+    int n_items, n_pairs;  // pairs per kv head: ceil(hpg / 2)
+    const int32_t *mask;
+    __nv_bfloat16 *out;
+    float scale_log2;      // logit scale times log2(e)
+};
+
+__device__ __forceinline__ bool wait(unsigned bar, unsigned parity, Tail *tl, unsigned code) {
+    return mbar_wait_bounded(bar, parity, &tl->abort_flag, &g_attn_status[0], &g_attn_status[1], code);
 }
+
+// The pair a CTA works on in its n-th round, and its two mask rows.
+struct Item {
+    int b, kvh, qb, h0, R;
+    const int32_t *m0, *m1;
+};
+
+__device__ __forceinline__ Item decode_item(const Params &P, int id) {
+    const Geom &g = P.g;
+    Item it;
+    const int per_qb = g.batch * g.G * P.n_pairs;
+    it.qb = g.n_qb - 1 - id / per_qb;  // late query blocks (most kept blocks under a causal mask) first
+    int rem = id % per_qb;
+    const int pair = rem % P.n_pairs;
+    rem /= P.n_pairs;
+    it.kvh = rem % g.G;
+    it.b = rem / g.G;
+    it.h0 = it.kvh * g.hpg + pair * 2;
+    it.R = min(2, g.hpg - pair * 2);
+    it.m0 = P.mask + (((long long)it.b * g.H + it.h0) * g.n_qb + it.qb) * g.k_top;
+    it.m1 = it.R == 2 ? it.m0 + (long long)g.n_qb * g.k_top : it.m0;
+    return it;
+}
+
+// Entry e of the two rows: key block per row (negative = this row has nothing at e). An entry
+// is processed if either row has a block there.
+struct Entry { int a, b; };
+__device__ __forceinline__ Entry load_entry(const Item &it, int e) {
+    Entry x;
+    x.a = __ldg(it.m0 + e);
+    x.b = it.R == 2 ? __ldg(it.m1 + e) : -1;
+    return x;
+}
+__device__ __forceinline__ int next_entry(const Item &it, int e, int k_top, Entry *x) {
+    for (++e; e < k_top; ++e) {
+        *x = load_entry(it, e);
+        if (x->a >= 0 || x->b >= 0) return e;
+    }
+    return k_top;
+}
+
+// ----------------------------------------------------------------------------------------------
+// Roles. All three walk the kept entries x_0 .. x_{n-1} of a pair in "rounds": round r handles
+// the logits of x_r and the P V product of x_{r-1}.
+// ----------------------------------------------------------------------------------------------
+__device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUtensorMap *tk, const CUtensorMap *tv,
+                              Tail *tl, unsigned q_smem, unsigned k_smem, unsigned v_smem) {
+    const Geom &g = P.g;
+    Ring ks, vs;
+    unsigned q_par = 0;
+    auto load_pair = [&](const CUtensorMap *map, unsigned dst, unsigned bar, const Item &it, Entry x) {
+        // a row without a block at this entry gets block 0; its logits are masked out entirely
+        const int ba = x.a >= 0 ? x.a : 0, bb = x.b >= 0 ? x.b : 0;
+        mbar_arrive_expect_tx(bar, (unsigned)kOperand);
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+            tma_load_4d(dst + c * 2 * kHalfTile, map, bar, c * 64, ba * kBlk, it.kvh, it.b);
+            tma_load_4d(dst + c * 2 * kHalfTile + kHalfTile, map, bar, c * 64, bb * kBlk, it.kvh, it.b);
+        }
+    };
+    for (int id = blockIdx.x; id < P.n_items; id += gridDim.x) {
+        const Item it = decode_item(P, id);
+        Entry cur, prev;
+        int e = next_entry(it, -1, g.k_top, &cur);
+        if (e >= g.k_top) continue;  // nothing kept: only the softmax warps act (they write zeros)
+        bool q_loaded = false, have_prev = false;
+        while (e < g.k_top || have_prev) {
+            const bool have_cur = e < g.k_top;
+            if (have_cur) {
+                if (!wait(smem_u32(&tl->k_empty[ks.idx]), ks.phase ^ 1, tl, 101)) return;
+                load_pair(tk, k_smem + ks.idx * kOperand, smem_u32(&tl->k_full[ks.idx]), it, cur);
+                ks.advance(kKStages);
+            }
+            if (!q_loaded) {  // behind the pair's first K tiles, which do not depend on the Q buffer
+                if (!wait(smem_u32(&tl->q_empty), q_par ^ 1, tl, 102)) return;
+                q_par ^= 1;
+                const unsigned bar = smem_u32(&tl->q_full);
+                mbar_arrive_expect_tx(bar, (unsigned)kOperand);
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    tma_load_4d(q_smem + c * 2 * kHalfTile, tq, bar, c * 64, it.qb * kBlk, it.h0, it.b);
+                    tma_load_4d(q_smem + c * 2 * kHalfTile + kHalfTile, tq, bar, c * 64, it.qb * kBlk, it.h0 + it.R - 1, it.b);
+                }
+                q_loaded = true;
+            }
+            if (have_prev) {
+                if (!wait(smem_u32(&tl->v_empty[vs.idx]), vs.phase ^ 1, tl, 103)) return;
+                load_pair(tv, v_smem + vs.idx * kOperand, smem_u32(&tl->v_full[vs.idx]), it, prev);
+                vs.advance(kVStages);
+            }
+            prev = cur;
+            have_prev = have_cur;
+            if (have_cur) e = next_entry(it, e, g.k_top, &cur);
+        }
+    }
+}
+
+__device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned p_smem, unsigned k_smem, unsigned v_smem,
+                         unsigned tmem_base) {
+    const Geom &g = P.g;
+    Ring ks, vs, sb, ob;
+    unsigned q_par = 0, p_par = 0;
+    for (int id = blockIdx.x; id < P.n_items; id += gridDim.x) {
+        const Item it = decode_item(P, id);
+        Entry cur;
+        int e = next_entry(it, -1, g.k_top, &cur);
+        if (e >= g.k_top) continue;
+        if (!wait(smem_u32(&tl->q_full), q_par, tl, 201)) return;
+        q_par ^= 1;
+        bool have_prev = false;
+        while (e < g.k_top || have_prev) {
+            const bool have_cur = e < g.k_top;
+            if (have_cur) {  // S = [Q_0; Q_1] [K_a; K_b]^T
+                if (!wait(smem_u32(&tl->k_full[ks.idx]), ks.phase, tl, 202)) return;
+                if (!wait(smem_u32(&tl->s_empty[sb.idx]), sb.phase ^ 1, tl, 203)) return;
+                tc_fence_after();
+                const unsigned d_tmem = tmem_base + sb.idx * 128;
+                const unsigned b_base = k_smem + ks.idx * kOperand;
+#pragma unroll
+                for (int c = 0; c < 2; ++c)
+#pragma unroll
+                    for (int k4 = 0; k4 < 4; ++k4)
+                        tc_mma_bf16(d_tmem, smem_desc_sw128(q_smem + c * 2 * kHalfTile + k4 * 32, 16, 1024),
+                                    smem_desc_sw128(b_base + c * 2 * kHalfTile + k4 * 32, 16, 1024), kIdescQK, (c | k4) != 0);
+                tc_commit(smem_u32(&tl->s_full[sb.idx]));
+                tc_commit(smem_u32(&tl->k_empty[ks.idx]));
+                sb.advance(2);
+                ks.advance(kKStages);
+                e = next_entry(it, e, g.k_top, &cur);
+                if (e >= g.k_top) tc_commit(smem_u32(&tl->q_empty));  // that was the pair's last use of Q
+            }
+            if (have_prev) {  // O = P [V_a; V_b] of the entry before
+                if (!wait(smem_u32(&tl->p_full), p_par, tl, 204)) return;
+                p_par ^= 1;
+                if (!wait(smem_u32(&tl->v_full[vs.idx]), vs.phase, tl, 205)) return;
+                if (!wait(smem_u32(&tl->o_empty[ob.idx]), ob.phase ^ 1, tl, 206)) return;
+                tc_fence_after();
+                const unsigned d_tmem = tmem_base + 256 + ob.idx * 128;
+                const unsigned b_base = v_smem + vs.idx * kOperand;
+#pragma unroll
+                for (int s = 0; s < 8; ++s)  // 16 keys per step: P column half s / 4, V rows 16 s ..
+                    tc_mma_bf16(d_tmem, smem_desc_sw128(p_smem + (s >> 2) * 2 * kHalfTile + (s & 3) * 32, 16, 1024),
+                                smem_desc_sw128(b_base + s * 2048, 2 * kHalfTile, 1024), kIdescPV, s != 0);
+                tc_commit(smem_u32(&tl->o_full[ob.idx]));
+                tc_commit(smem_u32(&tl->v_empty[vs.idx]));
+                ob.advance(2);
+                vs.advance(kVStages);
+            }
+            have_prev = have_cur;
+        }
+    }
+}
+
+// o[0..127] = o * alpha + O, O being this thread's lane of a 128-column TMEM buffer.
+__device__ __forceinline__ void fold_output(float *o, float alpha, unsigned taddr) {
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        unsigned r[32];
+        tmem_ld_32x32_issue(taddr + c * 32, r);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) o[c * 32 + i] = fmaf(o[c * 32 + i], alpha, __uint_as_float(r[i]));
+    }
+}
+
+__device__ void softmax_role(const Params &P, Tail *tl, unsigned char *p_ptr, unsigned tmem_base, int t) {
+    const Geom &g = P.g;
+    const int lane = t & 31, half = t >> 6, mq = t & 63;
+    const unsigned lane_off = (unsigned)(t & ~31) << 16;
+    // this thread's row of the block-diagonal P operand: column half = its row of the pair
+    unsigned char *p_row = p_ptr + half * 2 * kHalfTile + (t >> 3) * 1024 + (t & 7) * 128;
+    const int sw = t & 7;
+    Ring sb, ob;
+    for (int id = blockIdx.x; id < P.n_items; id += gridDim.x) {
+        const Item it = decode_item(P, id);
+        const long long tq = (long long)it.qb * kBlk + mq;
+        const bool row_active = half < it.R && tq < g.T;
+        float o[kD];
+#pragma unroll
+        for (int i = 0; i < kD; ++i) o[i] = 0.f;
+        float m = -CUDART_INF_F, l = 0.f, alpha_prev = 1.f;
+        bool have_prev = false;
+        Entry cur;
+        int e = next_entry(it, -1, g.k_top, &cur);
+        while (e < g.k_top) {
+            // logits of this token against its row's key block
+            if (!wait(smem_u32(&tl->s_full[sb.idx]), sb.phase, tl, 301)) return;
+            tc_fence_after();
+            unsigned r[64];
+            const unsigned s_addr = tmem_base + sb.idx * 128 + half * 64 + lane_off;
+            tmem_ld_32x32_issue(s_addr, r);
+            tmem_ld_32x32_issue(s_addr + 32, r + 32);
+            tmem_ld_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&tl->s_empty[sb.idx]));
+            sb.advance(2);
+            // keys of the block this token may attend: a prefix of n_hi keys (inside T, not after it if causal)
+            const int blk = half ? cur.b : cur.a;
+            int n_hi = 0;
+            if (blk >= 0 && row_active) {
+                const long long k0 = (long long)blk * kBlk;
+                long long lim = g.T - k0;
+                if (g.causal) lim = min(lim, tq - k0 + 1);
+                n_hi = (int)max(0ll, min(lim, (long long)kBlk));
+            }
+            float mx = -CUDART_INF_F;
+            if (n_hi == kBlk) {
+#pragma unroll
+                for (int i = 0; i < 64; ++i) mx = fmaxf(mx, __uint_as_float(r[i]));
+            } else {
+#pragma unroll
+                for (int i = 0; i < 64; ++i) mx = fmaxf(mx, i < n_hi ? __uint_as_float(r[i]) : -CUDART_INF_F);
+            }
+            const float m_new = fmaxf(m, mx);
+            // with no key allowed so far m_new is -inf: every p is 0 and nothing is rescaled
+            const float shift = m_new == -CUDART_INF_F ? 0.f : -m_new * P.scale_log2;
+            const float alpha = m_new == m ? 1.f : exp2f((m - m_new) * P.scale_log2);
+            float sum = 0.f;
+            unsigned packed[32];
+#pragma unroll
+            for (int i = 0; i < 64; i += 2) {
+                float p0 = exp2f(fmaf(__uint_as_float(r[i]), P.scale_log2, shift));
+                float p1 = exp2f(fmaf(__uint_as_float(r[i + 1]), P.scale_log2, shift));
+                p0 = i < n_hi ? p0 : 0.f;
+                p1 = i + 1 < n_hi ? p1 : 0.f;
+                sum += p0 + p1;
+                __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+                packed[i >> 1] = *reinterpret_cast<unsigned *>(&pk);
+            }
+            l = l * alpha + sum;
+            m = m_new;
+            // the P buffer is free, and the previous product ready, once the previous P V chain is done
+            if (have_prev) {
+                if (!wait(smem_u32(&tl->o_full[ob.idx]), ob.phase, tl, 302)) return;
+                tc_fence_after();
+            }
+#pragma unroll
+            for (int c = 0; c < 8; ++c)
+                *reinterpret_cast<uint4 *>(p_row + ((c ^ sw) << 4)) =
+                    make_uint4(packed[4 * c], packed[4 * c + 1], packed[4 * c + 2], packed[4 * c + 3]);
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&tl->p_full));
+            if (have_prev) {
+                fold_output(o, alpha_prev, tmem_base + 256 + ob.idx * 128 + lane_off);
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&tl->o_empty[ob.idx]));
+                ob.advance(2);
+            }
+            alpha_prev = alpha;
+            have_prev = true;
+            e = next_entry(it, e, g.k_top, &cur);
+        }
+        if (have_prev) {
+            if (!wait(smem_u32(&tl->o_full[ob.idx]), ob.phase, tl, 303)) return;
+            tc_fence_after();
+            fold_output(o, alpha_prev, tmem_base + 256 + ob.idx * 128 + lane_off);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&tl->o_empty[ob.idx]));
+            ob.advance(2);
+        }
+        if (row_active) {
+            const float inv = l > 0.f ? 1.f / l : 0.f;
+            uint4 *dst = reinterpret_cast<uint4 *>(P.out + (((long long)it.b * g.H + it.h0 + half) * g.T + tq) * kD);
+#pragma unroll
+            for (int c = 0; c < 16; ++c) {
+                unsigned w[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    __nv_bfloat162 pk = __floats2bfloat162_rn(o[8 * c + 2 * j] * inv, o[8 * c + 2 * j + 1] * inv);
+                    w[j] = *reinterpret_cast<unsigned *>(&pk);
+                }
+                dst[c] = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+               const __grid_constant__ CUtensorMap tmap_v, Params P) {
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    unsigned char *smem = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const unsigned q_smem = smem_u32(smem), p_smem = q_smem + kOperand, k_smem = p_smem + kOperand,
+                   v_smem = k_smem + kKStages * kOperand;
+    Tail *tl = (Tail *)(smem + (2 + kKStages + kVStages) * kOperand);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&tl->q_full), 1);
+        mbar_init(smem_u32(&tl->q_empty), 1);
+        for (int i = 0; i < kKStages; ++i) { mbar_init(smem_u32(&tl->k_full[i]), 1); mbar_init(smem_u32(&tl->k_empty[i]), 1); }
+        for (int i = 0; i < kVStages; ++i) { mbar_init(smem_u32(&tl->v_full[i]), 1); mbar_init(smem_u32(&tl->v_empty[i]), 1); }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(smem_u32(&tl->s_full[i]), 1); mbar_init(smem_u32(&tl->s_empty[i]), 4);
+            mbar_init(smem_u32(&tl->o_full[i]), 1); mbar_init(smem_u32(&tl->o_empty[i]), 4);
+        }
+        mbar_init(smem_u32(&tl->p_full), 4);
+        tl->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // P starts as zeros: its off-diagonal quadrants are never written again
+    for (int i = threadIdx.x; i < kOperand / 16; i += kThreads)
+        reinterpret_cast<uint4 *>(smem + kOperand)[i] = make_uint4(0, 0, 0, 0);
+    fence_async_smem();
+    if (warp == 1) tmem_alloc_512(smem_u32(&tl->tmem_base));  // all columns: one CTA per SM
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const unsigned tmem_base = tl->tmem_base;
+
+    if (warp == 0) {
+        if (lane == 0) producer_role(P, &tmap_q, &tmap_k, &tmap_v, tl, q_smem, k_smem, v_smem);
+    } else if (warp == 1) {
+        if (lane == 0) mma_role(P, tl, q_smem, p_smem, k_smem, v_smem, tmem_base);
+    } else if (warp >= 4) {
+        softmax_role(P, tl, smem + kOperand, tmem_base, (int)threadIdx.x - 128);
+    }
+    __syncwarp();
+
+    // Teardown. After an abort, copies and MMAs may still be in flight: leave them a bounded time
+    // to land before shared memory and TMEM are given back.
+    if (*(volatile int *)&tl->abort_flag) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < (1ll << 22)) { }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_512(tmem_base);
+    }
+}
+
+}  // namespace
+
+bool attn_tc_supported(const Geom &g, int dtype) {
+    return dtype == STREAM_BF16 && g.d == kD && g.bq == kBlk && g.bk == kBlk && tma_strides_ok(g);
+}
+
+stream_status launch_attn_tc(const Geom &g, const void *q, const void *k, const void *v, const int32_t *mask,
+                             float scale, void *out, cudaStream_t st) {
+    if ((((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)out) & 15) != 0) {
+        set_error("tensor-core attention kernel needs 16-byte aligned q, k, v and out");
+        return STREAM_ERR_UNSUPPORTED;
+    }
+    CUtensorMap tq, tk, tv;
+    stream_status rc = make_map_bf16_d128(&tq, q, g.T, g.H, g.batch, g.qs_t, g.qs_h, g.qs_b, "q");
+    if (rc != STREAM_OK) return rc;
+    rc = make_map_bf16_d128(&tk, k, g.T, g.G, g.batch, g.ks_t, g.ks_h, g.ks_b, "k");
+    if (rc != STREAM_OK) return rc;
+    rc = make_map_bf16_d128(&tv, v, g.T, g.G, g.batch, g.ks_t, g.ks_h, g.ks_b, "v");
+    if (rc != STREAM_OK) return rc;
+    Params P;
+    P.g = g;
+    P.n_pairs = (g.hpg + 1) / 2;
+    const long long n_items = (long long)g.batch * g.G * g.n_qb * P.n_pairs;
+    P.n_items = (int)n_items;
+    P.mask = mask;
+    P.out = (__nv_bfloat16 *)out;
+    P.scale_log2 = scale * 1.4426950408889634f;
+    const int n_sm = sm_count();
+    if (n_sm <= 0) { set_error("cannot read the SM count of the current device"); return STREAM_ERR_CUDA; }
+    cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(attn_tc)");
+    const int grid = (int)(n_items < n_sm ? n_items : n_sm);
+    attn_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(tq, tk, tv, P);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "attn_tc launch");
+    return STREAM_OK;
+}
+
+stream_status read_attn_status(unsigned int out[2], cudaStream_t st) {
+    cudaError_t e = cudaMemcpyFromSymbolAsync(out, g_attn_status, 2 * sizeof(unsigned int), 0, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpyFromSymbolAsync(attention status)");
+    e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+    return STREAM_OK;
+}
+
 }  // namespace stream

@@ -47,6 +47,8 @@ stream_status launch_mask_tc(const Geom &g, const void *q, const void *k, int32_
 bool attn_tc_supported(const Geom &g, int dtype);
 stream_status launch_attn_tc(const Geom &g, const void *q, const void *k, const void *v, const int32_t *mask,
                              float scale, void *out, cudaStream_t st);
+// Drains `st` and copies the tensor-core attention kernel's status words (code, block) to out.
+stream_status read_attn_status(unsigned int out[2], cudaStream_t st);
 
 __device__ __forceinline__ float to_float(float x) { return x; }
 __device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }

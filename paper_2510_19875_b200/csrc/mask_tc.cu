@@ -16,13 +16,14 @@
 // (level 1: stage-major, row-minor; later levels: row-major), synchronised by mbarriers only.
 // Every wait is bounded: on a timeout the CTA records an error code in the workspace header,
 // raises a shared abort flag, drains its own copies and leaves.
-#include <cuda.h>
 #include <math_constants.h>
 
-#include "common.cuh"
+#include "tc_common.cuh"
 
 namespace stream {
 namespace {
+
+using namespace tc;
 
 constexpr int kThreads = 256;
 constexpr int kR = 4;          // rows (query heads) per group
@@ -33,7 +34,6 @@ constexpr int kHalfTile = kBlk * 128;          // 64 rows x 128 bytes (one 64-ch
 constexpr int kStageBytes = 4 * kHalfTile;     // [2 channel halves][2 tiles]
 constexpr int kQBytes = 2 * kR * kHalfTile;    // [2 channel halves][kR rows]
 constexpr int kMaxJobs = 64;
-constexpr long long kWaitCycles = 1ll << 31;   // ~1 s: far beyond any legitimate wait
 
 struct Tail {
     unsigned long long full[kStages], empty[kStages], tmem_full[kSlots], tmem_empty[kSlots];
@@ -49,101 +49,16 @@ struct Tail {
 };
 constexpr int kSmemBytes = kQBytes + kStages * kStageBytes + (int)sizeof(Tail) + 1024;
 
-// ----------------------------------------------------------------------------------------------
-// PTX wrappers
-// ----------------------------------------------------------------------------------------------
-__device__ __forceinline__ unsigned smem_u32(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(unsigned bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(unsigned bar, unsigned bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
-    unsigned ok;
-    asm volatile(
-        "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
+// Bounded wait that reports into the workspace header; false means the CTA is aborting.
+__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, Tail *tl, WorkspaceHeader *ws, unsigned code) {
+    return mbar_wait_bounded(bar, parity, &tl->abort_flag, &ws->error, &ws->error_info, code);
 }
 
-// Bounded wait. Returns false if the CTA is aborting (or this wait ran out, which starts an abort).
-__device__ __noinline__ bool mbar_wait(unsigned bar, unsigned parity, Tail *tl, WorkspaceHeader *ws, unsigned code) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    for (;;) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (*(volatile int *)&tl->abort_flag) return false;
-        if (clock64() - t0 > kWaitCycles) {
-            *(volatile int *)&tl->abort_flag = 1;
-            if (atomicCAS(&ws->error, 0u, code) == 0u) ws->error_info = blockIdx.x;
-            return false;
-        }
-    }
-}
+// K-major, 128-byte-swizzled operand with 8-row groups 1024 bytes apart.
+__device__ __forceinline__ unsigned long long smem_desc(unsigned addr) { return smem_desc_sw128(addr, 16, 1024); }
 
-__device__ __forceinline__ void tma_load_4d(unsigned dst, const CUtensorMap *map, unsigned bar, int c0, int c1, int c2,
-                                            int c3) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-        ::"r"(dst), "l"((unsigned long long)map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
-        : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tc_commit(unsigned bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-
-__device__ __forceinline__ void tc_mma_bf16(unsigned d_tmem, unsigned long long adesc, unsigned long long bdesc,
-                                            unsigned idesc, unsigned accumulate) {
-    asm volatile(
-        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-
-// 32 lanes x 32 consecutive fp32 columns of TMEM: thread i gets lane (base lane + i).
-__device__ __forceinline__ void tmem_ld_32x32(unsigned taddr, float *v) {
-    unsigned r[32];
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr)
-        : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-}
-
-__device__ __forceinline__ float warp_max(float x) {
-    float r;
-    asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(x));
-    return r;
-}
-
-// Shared-memory matrix descriptor: K-major rows of 128 bytes, 128-byte swizzle, 8-row groups
-// 1024 bytes apart, descriptor version 1 (sm_100).
-__device__ __forceinline__ unsigned long long smem_desc(unsigned addr) {
-    return (unsigned long long)((addr >> 4) & 0x3FFF) | (1ull << 16) | ((unsigned long long)(1024 >> 4) << 32) |
-           (1ull << 46) | (2ull << 61);
-}
-
-// kind::f16 instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = 64.
-constexpr unsigned kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
+// D fp32, A and B bf16, both K-major, M = 128, N = 64.
+constexpr unsigned kIdesc = idesc_bf16(128, 64, false);
 
 struct Params {
     Geom g;
@@ -156,14 +71,6 @@ struct Params {
 // ----------------------------------------------------------------------------------------------
 // Roles
 // ----------------------------------------------------------------------------------------------
-struct Ring {  // position in a ring of barriers with phase tracking
-    int idx = 0;
-    unsigned phase = 0;
-    __device__ void advance(int n) {
-        if (++idx == n) { idx = 0; phase ^= 1; }
-    }
-};
-
 __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUtensorMap *tk, Tail *tl, unsigned q_smem,
                               unsigned k_smem) {
     const Geom &g = P.g;
@@ -455,12 +362,10 @@ mask_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         for (int i = 0; i < kR; ++i) mbar_init(smem_u32(&tl->scores_done[i]), 4);
         tl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        fence_async_smem();
     }
     if (warp == 1) {  // TMEM: all 512 columns (one CTA per SM)
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tl->tmem_base)), "r"(512)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        tmem_alloc_512(smem_u32(&tl->tmem_base));
     }
     tc_fence_before();
     __syncthreads();
@@ -488,54 +393,18 @@ mask_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+        tmem_dealloc_512(tmem_base);
     }
 }
 
 // ----------------------------------------------------------------------------------------------
 // Host side
 // ----------------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (fn == nullptr) {
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = (EncodeTiledFn)p;
-    }
-    return fn;
-}
-
-// [batch, heads, T, 128] bf16 with element strides -> 4-D map with a 64 x 64 box, 128-byte swizzle.
-stream_status make_map(CUtensorMap *map, const void *base, long long T, int heads, int batch, long long s_t,
-                       long long s_h, long long s_b, const char *what) {
-    EncodeTiledFn fn = encode_fn();
-    if (fn == nullptr) { set_error("cuTensorMapEncodeTiled is not available from this driver"); return STREAM_ERR_CUDA; }
-    // extents of 1 may come with arbitrary strides: give them a well-formed one
-    if (heads == 1) s_h = s_t * T;
-    if (batch == 1) s_b = s_h * heads;
-    cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)T, (cuuint64_t)heads, (cuuint64_t)batch};
-    cuuint64_t strides[3] = {(cuuint64_t)s_t * 2, (cuuint64_t)s_h * 2, (cuuint64_t)s_b * 2};
-    cuuint32_t box[4] = {64, 64, 1, 1}, estr[4] = {1, 1, 1, 1};
-    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled(%s) failed with %d", what, (int)r); return STREAM_ERR_CUDA; }
-    return STREAM_OK;
-}
-
 }  // namespace
 
 bool mask_tc_supported(const Geom &g, int dtype) {
-    auto ok_stride = [](long long s) { return s % 8 == 0; };  // 16-byte multiples for TMA
     return dtype == STREAM_BF16 && g.d == kD && g.bq == kBlk && g.bk == kBlk && g.k_top <= 32 && g.levels >= 1 &&
-           ok_stride(g.qs_t) && ok_stride(g.qs_h) && ok_stride(g.qs_b) && ok_stride(g.ks_t) && ok_stride(g.ks_h) &&
-           ok_stride(g.ks_b);
+           tma_strides_ok(g);
 }
 
 stream_status launch_mask_tc(const Geom &g, const void *q, const void *k, int32_t *mask, float *score,
@@ -545,9 +414,9 @@ stream_status launch_mask_tc(const Geom &g, const void *q, const void *k, int32_
         return STREAM_ERR_UNSUPPORTED;
     }
     CUtensorMap tq, tk;
-    stream_status rc = make_map(&tq, q, g.T, g.H, g.batch, g.qs_t, g.qs_h, g.qs_b, "q");
+    stream_status rc = make_map_bf16_d128(&tq, q, g.T, g.H, g.batch, g.qs_t, g.qs_h, g.qs_b, "q");
     if (rc != STREAM_OK) return rc;
-    rc = make_map(&tk, k, g.T, g.G, g.batch, g.ks_t, g.ks_h, g.ks_b, "k");
+    rc = make_map_bf16_d128(&tk, k, g.T, g.G, g.batch, g.ks_t, g.ks_h, g.ks_b, "k");
     if (rc != STREAM_OK) return rc;
     Params P;
     P.g = g;
@@ -555,13 +424,8 @@ stream_status launch_mask_tc(const Geom &g, const void *q, const void *k, int32_
     long long n_groups = (long long)g.batch * g.G * g.n_qb * P.n_chunks;
     P.n_groups = (int)n_groups;
     P.mask = mask; P.score = score; P.ws = ws;
-    static int n_sm = 0;
-    if (n_sm == 0) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaError_t e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
-        if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
-    }
+    const int n_sm = sm_count();
+    if (n_sm <= 0) { set_error("cannot read the SM count of the current device"); return STREAM_ERR_CUDA; }
     cudaError_t e = cudaFuncSetAttribute(mask_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(mask_tc)");
     int grid = (int)(n_groups < n_sm ? n_groups : n_sm);

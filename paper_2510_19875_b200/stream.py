@@ -80,6 +80,8 @@ def _load():
     lib.stream_sparse_attention.argtypes = [P, vp, vp, vp, vp, ctypes.c_float, vp, vp]
     lib.stream_read_stats.restype = ctypes.c_int
     lib.stream_read_stats.argtypes = [vp, ctypes.POINTER(StreamStats), vp]
+    lib.stream_check_device_status.restype = ctypes.c_int
+    lib.stream_check_device_status.argtypes = [vp]
     lib.stream_host_staging_bytes.restype = sz
     lib.stream_host_staging_bytes.argtypes = [P]
     lib.stream_run_host.restype = ctypes.c_int
@@ -142,6 +144,11 @@ def stream_read_stats(workspace, stream=None) -> StreamStats:
     st = StreamStats()
     _raise(_load().stream_read_stats(_addr(workspace), ctypes.byref(st), _stream_handle(stream)))
     return st
+
+
+def stream_check_device_status(stream=None) -> None:
+    """Drains the stream; raises if a kernel without a workspace recorded a bounded wait that ran out."""
+    _raise(_load().stream_check_device_status(_stream_handle(stream)))
 
 
 def stream_host_staging_bytes(p: StreamProblem) -> int:

@@ -195,6 +195,53 @@ def test_attention_generic_unequal_blocks_and_non_causal(S):
     attention_parity(S, w, None, impl="generic", causal=False)
 
 
+ATTN_TC_CASES = [
+    dict(),                                                   # two pairs of one kv head
+    dict(T=2048, k_top=16, n_q_heads=8, n_kv_heads=2),
+    dict(T=5000, k_top=5, n_q_heads=7, n_kv_heads=1),         # ragged T, an odd head left alone in its pair
+    dict(T=3000, k_top=3, n_q_heads=6, n_kv_heads=2, batch=2, local=True),
+    dict(T=1024, k_top=32, n_q_heads=4, n_kv_heads=4),        # full causal mask, one head per kv head
+    dict(T=100, k_top=4, n_q_heads=4, n_kv_heads=2),          # two key blocks, ragged
+    dict(T=8192, k_top=32, n_q_heads=8, n_kv_heads=2, anchors=True),
+]
+
+
+@pytest.mark.parametrize("kw", ATTN_TC_CASES)
+def test_attention_tensor_core_small(S, kw):
+    w = wl.generate(tc_spec(**kw))
+    attention_parity(S, w, None, impl="tensor")
+    S.stream_check_device_status()
+
+
+def test_attention_tensor_core_non_causal(S):
+    w = wl.generate(tc_spec(T=3000, k_top=6))
+    attention_parity(S, w, None, impl="tensor", causal=False)
+
+
+@pytest.mark.parametrize("impl", ["tensor", "generic"])
+@pytest.mark.parametrize("causal", [True, False])
+def test_attention_arbitrary_mask(S, impl, causal):
+    """Any int32 mask is legal input: unsorted, with holes, rows of unequal length, blocks after the
+    query (all their keys are excluded under a causal C), rows with nothing kept (zeros)."""
+    spec = tc_spec(T=2500, k_top=6, n_q_heads=6, n_kv_heads=2, batch=2)
+    w = wl.generate(spec)
+    p = oracle_problem(spec, causal=causal)
+    nqb, rng = spec.n_blocks, np.random.default_rng(11)
+    mask = rng.integers(0, nqb, size=(spec.n_rows, spec.k_top)).astype(np.int32)
+    mask[rng.random(mask.shape) < 0.35] = -1
+    mask[rng.random(spec.n_rows) < 0.1] = -1
+    q, k, v = w.torch_tensors("cuda")
+    mask_dev = torch.from_numpy(mask.reshape(spec.batch, spec.n_q_heads, nqb, spec.k_top)).cuda()
+    out = S.sparse_attention(q, k, v, mask_dev, block_q=64, block_k=64, causal=causal, impl=impl)
+    torch.cuda.synchronize()
+    ref = so.sparse_attention_rows(p, w.q, w.k, w.v, mask, None)
+    got = out.float().cpu().numpy().reshape(spec.batch * spec.n_q_heads, spec.T, spec.d)
+    for rid in range(spec.n_rows):
+        bh, qb = divmod(rid, nqb)
+        lo, hi = qb * 64, min(spec.T, qb * 64 + 64)
+        assert np.abs(got[bh, lo:hi] - ref[rid, : hi - lo]).max() <= ATTN_TOL["bf16"], rid
+
+
 def test_full_mask_attention_equals_dense_softmax_attention(S):
     """k covers every causal block: the sparse pass must reproduce dense causal attention."""
     w = wl.generate(small_spec(dtype="bf16", d=128, block=64, T=1024, k_top=16, n_q_heads=4, n_kv_heads=2))

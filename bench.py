@@ -123,15 +123,57 @@ def hbm_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
-def ncu_traffic(kernel_key: str, units: int):
-    """DRAM bytes per launch from the committed ncu summary, scaled by the units processed."""
+KERNEL_SOURCES = {
+    "mask_tc_kernel": ("mask_tc.cu", "tc_common.cuh", "common.cuh"),
+    "attn_tc_kernel": ("attn_tc.cu", "tc_common.cuh", "common.cuh"),
+}
+
+
+def kernel_source_hash(kernel: str) -> str:
+    """Hash of the sources a kernel is built from; a stored ncu figure is only valid for the same hash."""
+    import hashlib
+
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES[kernel]:
+        with open(os.path.join(ROOT, "paper_2510_19875_b200", "csrc", name), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(kernel: str, spec):
+    """DRAM bytes (read + write) per launch of `kernel` on this workload from the committed ncu
+    capture, or None if there is none for this workload and T or the kernel's sources changed since."""
     path = os.path.join(ROOT, "profiles", "dram_traffic.json")
     try:
         with open(path) as fh:
-            rec = json.load(fh)[kernel_key]
-        return rec["dram_bytes_per_unit"] * units
+            rec = json.load(fh)[kernel]
+        if rec["source_hash"] != kernel_source_hash(kernel) or rec["workload"] != spec.name or rec["T"] != spec.T:
+            return None
+        return float(rec["dram_bytes_per_launch"])
     except (OSError, KeyError, ValueError):
         return None
+
+
+def rank_env():
+    """(world size, rank, local rank) as torchrun exports them; (1, 0, 0) when run directly."""
+    return (int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("RANK", "0")),
+            int(os.environ.get("LOCAL_RANK", "0")))
+
+
+def max_over_ranks(values, device):
+    """Element-wise maximum over the ranks of a list of floats (the slowest rank sets the time)."""
+    import torch
+    import torch.distributed as dist
+
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def job_value(world: int, units_per_rank: int, steps: int, total_ms: float) -> float:
+    """Whole-job throughput: every rank processes `units_per_rank` per step (weak scaling)."""
+    return world * units_per_rank * steps / (total_ms * 1e-3)
 
 
 def oracle_sample_rate(spec, w, seconds: float):
@@ -161,8 +203,7 @@ def oracle_sample_rate(spec, w, seconds: float):
 
 def run_reference(args):
     """The oracle as the reference arm: each step is a bounded row sample of the same workload."""
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    if rank_env()[1] != 0:
         return
     import numpy as np
 
@@ -209,9 +250,7 @@ def run_ours(args):
     from paper_2510_19875_b200 import stream as S
     from paper_2510_19875_b200 import workloads as wl
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world, rank, local = rank_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: there is no CPU path for the library")
     torch.cuda.set_device(local)
@@ -290,10 +329,7 @@ def run_ours(args):
                "h2d": qp.numel() * qp.element_size() + 2 * kp.numel() * kp.element_size(),
                "d2h": mask_host.numel() * 4 + out_host.numel() * out_host.element_size()}
 
-    times = torch.tensor([total_ms, mask_ms, attn_ms, e2e["ms"] if e2e else 0.0], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    total_ms, mask_ms, attn_ms, e2e_ms = times.tolist()
+    total_ms, mask_ms, attn_ms, e2e_ms = max_over_ranks([total_ms, mask_ms, attn_ms, e2e["ms"] if e2e else 0.0], dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -302,23 +338,39 @@ def run_ours(args):
     units = spec.batch * spec.n_q_heads * spec.T  # query-token-heads per rank per step
     esz = 2 if spec.dtype == "bf16" else 4
     S_tiles = int(stats.tiles_scored)
-    alg_bytes = S_tiles * spec.block * spec.d * esz + units * spec.d * esz + spec.n_rows * spec.k_top * 4
+    tile_bytes = spec.block * spec.d * esz
     peak, peak_kind = hbm_peak()
-    achieved = alg_bytes / (mask_ms * 1e-3) / 1e9
-    traffic = ncu_traffic("stream_build_mask", units)
-    attn_bytes = kept * 2 * spec.block * spec.d * esz + 2 * units * spec.d * esz
+    tc = spec.dtype == "bf16" and spec.d == 128 and spec.block == 64 and args.kernels != "generic"
+    # algorithmic bytes per launch: every scored / kept tile counted as one fetch, Q in, result out
+    kernels = {
+        "stream_build_mask": {
+            "kernel": "mask_tc_kernel" if tc and spec.k_top <= 32 else "mask_generic_kernel", "ms": mask_ms,
+            "algorithmic_bytes": S_tiles * tile_bytes + units * spec.d * esz + spec.n_rows * spec.k_top * 4,
+            "tiles_scored": S_tiles, "value": units / (mask_ms * 1e-3), "unit": UNIT,
+            "tensor_tflops": S_tiles * 2.0 * spec.block * spec.block * spec.d / (mask_ms * 1e-3) / 1e12},
+        "stream_sparse_attention": {
+            "kernel": "attn_tc_kernel" if tc else "attn_generic_kernel", "ms": attn_ms,
+            "algorithmic_bytes": kept * 2 * tile_bytes + 2 * units * spec.d * esz, "kept_blocks": kept,
+            "tensor_tflops": kept * 4.0 * spec.block * spec.block * spec.d / (attn_ms * 1e-3) / 1e12},
+    }
+    for rec in kernels.values():
+        rec["algorithmic_gbs"] = rec["algorithmic_bytes"] / (rec["ms"] * 1e-3) / 1e9
+        rec["frac_of_hbm_peak"] = rec["algorithmic_gbs"] / peak
+    dominant = max(kernels, key=lambda n: kernels[n]["ms"])
+    dom = kernels[dominant]
     line = {
-        "metric": METRIC, "value": world * units * args.steps / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world,
+        "metric": METRIC, "value": job_value(world, units, args.steps, total_ms), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": spec.dtype, "data": "synthetic",
         "config": workload_config(spec, {"l2": "inputs larger than L2 (Q+K+V %.0f MiB per step)" % (
             (q.numel() + 2 * k.numel()) * esz / 2**20), "kernels": args.kernels, "per_rank": "one independent layer each"}),
-        "mask_build": {"ms": mask_ms, "value": units / (mask_ms * 1e-3), "unit": UNIT, "tiles_scored": S_tiles,
-                       "tensor_tflops": S_tiles * 2.0 * spec.block * spec.block * spec.d / (mask_ms * 1e-3) / 1e12},
-        "sparse_attention": {"ms": attn_ms, "kept_blocks": kept, "algorithmic_gbs": attn_bytes / (attn_ms * 1e-3) / 1e9},
-        "roofline": {"kernel": "stream_build_mask", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "traffic": traffic, "peak_kind": f"of {peak_kind}",
-                     "algorithmic_bytes": alg_bytes, "frac_of_8TBs_nominal": achieved / 8000.0},
+        "mask_build": kernels["stream_build_mask"], "sparse_attention": kernels["stream_sparse_attention"],
+        "roofline": {"kernel": dom["kernel"], "entry_point": dominant, "bound": "hbm", "achieved": dom["algorithmic_gbs"],
+                     "peak": peak, "unit": "GB/s", "frac": dom["algorithmic_gbs"] / peak,
+                     "traffic": ncu_traffic(dom["kernel"], spec) if dom["kernel"] in KERNEL_SOURCES else None,
+                     "peak_kind": f"of {peak_kind}", "algorithmic_bytes": dom["algorithmic_bytes"],
+                     "share_of_step": dom["ms"] / (mask_ms + attn_ms),
+                     "frac_of_8TBs_nominal": dom["algorithmic_gbs"] / 8000.0},
         "clocks": clocks,
         "gpu_launches": 2 * args.steps,
     }

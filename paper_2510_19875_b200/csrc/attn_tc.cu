@@ -3,11 +3,11 @@
 //
 // One persistent CTA per SM works through "pairs": two query heads of one kv head at one query
 // block. Their Q tiles are stacked into one 128-row A operand. For every mask entry e the two
-// rows name one key block each (K_a, K_b, usually different); their tiles are fetched by TMA
-// (128-byte swizzle) and stacked too, so that
-//     S = [Q_0; Q_1] [K_a; K_b]^T      (128 x 128, fp32 in TMEM)
-// holds row 0's logits in its upper-left quadrant and row 1's in its lower-right one. The four
-// softmax warps own one TMEM lane (= one query token) per thread: they read their 64 logits,
+// rows name one key block each (K_a, K_b, usually different); each tile arrives by one TMA box
+// (128-byte swizzle) and
+//     S = [Q_0; Q_1] [K_a; K_b]^T      (128 x 128, fp32 in TMEM; one N = 64 chain per tile)
+// holds row 0's logits in its upper-left quadrant and row 1's in its lower-right one. The
+// softmax warps own one TMEM lane (= one query token) per thread pair: they read its 64 logits,
 // apply the element-level mask C, update the running maximum and sum (online softmax, fp32), and
 // write P = exp(.) as bf16 into a block-diagonal 128 x 128 A operand in shared memory whose
 // off-diagonal quadrants stay zero. Then
@@ -16,10 +16,12 @@
 // output registers (o = o * alpha + O_e) one iteration later, so that the tensor core works on
 // the next logits meanwhile.
 //
-// Roles (256 threads): warp 0 TMA producer, warp 1 MMA issuer + TMEM owner, warps 4..7 softmax.
-// Every role derives the same sequence of (pair, entry) from blockIdx and the mask itself; they
-// meet only on mbarriers. Every wait is bounded: on a timeout the CTA records a code in a device
-// status word, raises a shared abort flag, lets its copies drain and leaves.
+// Roles (384 threads): warp 0 TMA producer, warp 1 MMA issuer + TMEM owner, warp 2 copies the
+// pairs' mask rows from global to shared memory ahead of everyone else, warps 4..11 softmax (two
+// threads per query token: half of its keys and half of its output channels each). Every role
+// walks the same sequence of (pair, entry), read from the shared copy of the mask rows; they meet
+// only on mbarriers. Every wait is bounded: on a timeout the CTA records a code in a device status
+// word, raises a shared abort flag, lets its copies drain and leaves.
 #include <math_constants.h>
 
 #include "tc_common.cuh"
@@ -34,24 +36,32 @@ namespace {
 
 using namespace tc;
 
-constexpr int kThreads = 256;
+constexpr int kThreads = 384;
 constexpr int kBlk = 64, kD = 128;
 constexpr int kHalfTile = kBlk * 128;       // 64 rows x 128 bytes
-constexpr int kOperand = 4 * kHalfTile;     // 128 rows x 256 bytes as [2 column halves][128 rows][128 B]
-constexpr int kKStages = 3, kVStages = 2;
+constexpr int kTile = 2 * kHalfTile;        // one 64 x 128 tile as [2 channel halves][64 rows][128 B]
+constexpr int kOperand = 2 * kTile;         // two tiles (K_a, K_b or V_a, V_b), or a 128-row operand
+constexpr int kKStages = 2, kVStages = 2;
+constexpr int kMaskSlots = 2;               // pairs whose mask rows are resident
+constexpr int kMaxKTopTc = 1024;
 
 struct Tail {
     unsigned long long q_full, q_empty;
     unsigned long long k_full[kKStages], k_empty[kKStages], v_full[kVStages], v_empty[kVStages];
     unsigned long long s_full[2], s_empty[2], o_full[2], o_empty[2], p_full;
+    unsigned long long m_full[kMaskSlots], m_empty[kMaskSlots];
+    unsigned long long x_bar[4];  // softmax warps w and w + 4 meet here
     unsigned int tmem_base;
     int abort_flag;
+    float xch[2][128][2];         // their exchange slots: [buffer][token][part]
+    int rows[kMaskSlots][2][kMaxKTopTc];  // mask rows of the resident pairs (-1 where a row has nothing)
 };
 constexpr int kSmemBytes = (2 + kKStages + kVStages) * kOperand + (int)sizeof(Tail) + 1024;
 static_assert(kSmemBytes <= 232448, "exceeds the shared memory of one CTA");
 
-constexpr unsigned kIdescQK = idesc_bf16(128, 128, false);  // B = stacked K tiles, K-major
+constexpr unsigned kIdescQK = idesc_bf16(128, 64, false);   // B = one K tile, K-major
 constexpr unsigned kIdescPV = idesc_bf16(128, 128, true);   // B = stacked V tiles, MN-major
+constexpr unsigned kHiK = desc_hi_sw128(1024);              // every operand: 8-row (8-key) groups 1024 bytes apart
 
 struct Params {
     Geom g;
@@ -65,10 +75,9 @@ __device__ __forceinline__ bool wait(unsigned bar, unsigned parity, Tail *tl, un
     return mbar_wait_bounded(bar, parity, &tl->abort_flag, &g_attn_status[0], &g_attn_status[1], code);
 }
 
-// The pair a CTA works on in its n-th round, and its two mask rows.
+// The pair a CTA works on in its n-th round.
 struct Item {
     int b, kvh, qb, h0, R;
-    const int32_t *m0, *m1;
 };
 
 __device__ __forceinline__ Item decode_item(const Params &P, int id) {
@@ -83,54 +92,64 @@ __device__ __forceinline__ Item decode_item(const Params &P, int id) {
     it.b = rem / g.G;
     it.h0 = it.kvh * g.hpg + pair * 2;
     it.R = min(2, g.hpg - pair * 2);
-    it.m0 = P.mask + (((long long)it.b * g.H + it.h0) * g.n_qb + it.qb) * g.k_top;
-    it.m1 = it.R == 2 ? it.m0 + (long long)g.n_qb * g.k_top : it.m0;
     return it;
 }
 
 // Entry e of the two rows: key block per row (negative = this row has nothing at e). An entry
-// is processed if either row has a block there.
+// is processed if either row has a block there. `rows` is the pair's shared copy [2][kMaxKTopTc].
 struct Entry { int a, b; };
-__device__ __forceinline__ Entry load_entry(const Item &it, int e) {
-    Entry x;
-    x.a = __ldg(it.m0 + e);
-    x.b = it.R == 2 ? __ldg(it.m1 + e) : -1;
-    return x;
-}
-__device__ __forceinline__ int next_entry(const Item &it, int e, int k_top, Entry *x) {
+__device__ __forceinline__ int next_entry(const int *rows, int e, int k_top, Entry *x) {
     for (++e; e < k_top; ++e) {
-        *x = load_entry(it, e);
+        x->a = rows[e];
+        x->b = rows[kMaxKTopTc + e];
         if (x->a >= 0 || x->b >= 0) return e;
     }
     return k_top;
 }
 
 // ----------------------------------------------------------------------------------------------
-// Roles. All three walk the kept entries x_0 .. x_{n-1} of a pair in "rounds": round r handles
-// the logits of x_r and the P V product of x_{r-1}.
+// Roles. All walk the kept entries x_0 .. x_{n-1} of a pair in "rounds": round r handles the
+// logits of x_r and the P V product of x_{r-1}.
 // ----------------------------------------------------------------------------------------------
+__device__ void mask_loader_role(const Params &P, Tail *tl, int lane) {
+    const Geom &g = P.g;
+    Ring ms;
+    for (int id = blockIdx.x; id < P.n_items; id += gridDim.x) {
+        const Item it = decode_item(P, id);
+        if (!wait(smem_u32(&tl->m_empty[ms.idx]), ms.phase ^ 1, tl, 401)) return;
+        const int32_t *m0 = P.mask + (((long long)it.b * g.H + it.h0) * g.n_qb + it.qb) * g.k_top;
+        const int32_t *m1 = m0 + (long long)g.n_qb * g.k_top;
+        int *dst = tl->rows[ms.idx][0];
+        for (int e = lane; e < g.k_top; e += 32) {
+            dst[e] = __ldg(m0 + e);
+            dst[kMaxKTopTc + e] = it.R == 2 ? __ldg(m1 + e) : -1;
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&tl->m_full[ms.idx]));
+        ms.advance(kMaskSlots);
+    }
+}
+
 __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUtensorMap *tk, const CUtensorMap *tv,
                               Tail *tl, unsigned q_smem, unsigned k_smem, unsigned v_smem) {
     const Geom &g = P.g;
-    Ring ks, vs;
+    Ring ks, vs, ms;
     unsigned q_par = 0;
     auto load_pair = [&](const CUtensorMap *map, unsigned dst, unsigned bar, const Item &it, Entry x) {
         // a row without a block at this entry gets block 0; its logits are masked out entirely
         const int ba = x.a >= 0 ? x.a : 0, bb = x.b >= 0 ? x.b : 0;
         mbar_arrive_expect_tx(bar, (unsigned)kOperand);
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
-            tma_load_4d(dst + c * 2 * kHalfTile, map, bar, c * 64, ba * kBlk, it.kvh, it.b);
-            tma_load_4d(dst + c * 2 * kHalfTile + kHalfTile, map, bar, c * 64, bb * kBlk, it.kvh, it.b);
-        }
+        tma_load_5d(dst, map, bar, 0, ba * kBlk, it.kvh, 0, it.b);
+        tma_load_5d(dst + kTile, map, bar, 0, bb * kBlk, it.kvh, 0, it.b);
     };
     for (int id = blockIdx.x; id < P.n_items; id += gridDim.x) {
         const Item it = decode_item(P, id);
+        if (!wait(smem_u32(&tl->m_full[ms.idx]), ms.phase, tl, 104)) return;
+        const int *rows = tl->rows[ms.idx][0];
         Entry cur, prev;
-        int e = next_entry(it, -1, g.k_top, &cur);
-        if (e >= g.k_top) continue;  // nothing kept: only the softmax warps act (they write zeros)
+        int e = next_entry(rows, -1, g.k_top, &cur);
         bool q_loaded = false, have_prev = false;
-        while (e < g.k_top || have_prev) {
+        while (e < g.k_top || have_prev) {  // (a pair with nothing kept: only the softmax warps act)
             const bool have_cur = e < g.k_top;
             if (have_cur) {
                 if (!wait(smem_u32(&tl->k_empty[ks.idx]), ks.phase ^ 1, tl, 101)) return;
@@ -142,11 +161,7 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
                 q_par ^= 1;
                 const unsigned bar = smem_u32(&tl->q_full);
                 mbar_arrive_expect_tx(bar, (unsigned)kOperand);
-#pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    tma_load_4d(q_smem + c * 2 * kHalfTile, tq, bar, c * 64, it.qb * kBlk, it.h0, it.b);
-                    tma_load_4d(q_smem + c * 2 * kHalfTile + kHalfTile, tq, bar, c * 64, it.qb * kBlk, it.h0 + it.R - 1, it.b);
-                }
+                tma_load_5d(q_smem, tq, bar, 0, it.qb * kBlk, it.h0, 0, it.b);  // heads h0 and h0 + 1
                 q_loaded = true;
             }
             if (have_prev) {
@@ -156,43 +171,54 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
             }
             prev = cur;
             have_prev = have_cur;
-            if (have_cur) e = next_entry(it, e, g.k_top, &cur);
+            if (have_cur) e = next_entry(rows, e, g.k_top, &cur);
         }
+        mbar_arrive(smem_u32(&tl->m_empty[ms.idx]));
+        ms.advance(kMaskSlots);
     }
 }
 
 __device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned p_smem, unsigned k_smem, unsigned v_smem,
                          unsigned tmem_base) {
     const Geom &g = P.g;
-    Ring ks, vs, sb, ob;
+    Ring ks, vs, sb, ob, ms;
     unsigned q_par = 0, p_par = 0;
+    // low descriptor words of the operand buffers; K-major ones ignore the leading offset, the
+    // MN-major V tiles have their two 64-channel halves kHalfTile apart
+    const unsigned q_lo = desc_lo_sw128(q_smem, 16), p_lo = desc_lo_sw128(p_smem, 16), k_lo = desc_lo_sw128(k_smem, 16),
+                   v_lo = desc_lo_sw128(v_smem, kHalfTile);
     for (int id = blockIdx.x; id < P.n_items; id += gridDim.x) {
-        const Item it = decode_item(P, id);
+        if (!wait(smem_u32(&tl->m_full[ms.idx]), ms.phase, tl, 207)) return;
+        const int *rows = tl->rows[ms.idx][0];
         Entry cur;
-        int e = next_entry(it, -1, g.k_top, &cur);
-        if (e >= g.k_top) continue;
-        if (!wait(smem_u32(&tl->q_full), q_par, tl, 201)) return;
-        q_par ^= 1;
+        int e = next_entry(rows, -1, g.k_top, &cur);
+        if (e < g.k_top) {
+            if (!wait(smem_u32(&tl->q_full), q_par, tl, 201)) return;
+            q_par ^= 1;
+        }
         bool have_prev = false;
         while (e < g.k_top || have_prev) {
             const bool have_cur = e < g.k_top;
-            if (have_cur) {  // S = [Q_0; Q_1] [K_a; K_b]^T
+            if (have_cur) {  // S = [Q_0; Q_1] [K_a; K_b]^T, one chain per K tile
                 if (!wait(smem_u32(&tl->k_full[ks.idx]), ks.phase, tl, 202)) return;
                 if (!wait(smem_u32(&tl->s_empty[sb.idx]), sb.phase ^ 1, tl, 203)) return;
                 tc_fence_after();
                 const unsigned d_tmem = tmem_base + sb.idx * 128;
-                const unsigned b_base = k_smem + ks.idx * kOperand;
+                const unsigned b_lo = k_lo + ks.idx * (kOperand >> 4);
 #pragma unroll
-                for (int c = 0; c < 2; ++c)
+                for (int tile = 0; tile < 2; ++tile)
 #pragma unroll
-                    for (int k4 = 0; k4 < 4; ++k4)
-                        tc_mma_bf16(d_tmem, smem_desc_sw128(q_smem + c * 2 * kHalfTile + k4 * 32, 16, 1024),
-                                    smem_desc_sw128(b_base + c * 2 * kHalfTile + k4 * 32, 16, 1024), kIdescQK, (c | k4) != 0);
+                    for (int c = 0; c < 2; ++c)
+#pragma unroll
+                        for (int k4 = 0; k4 < 4; ++k4)
+                            tc_mma_bf16_split(d_tmem + tile * 64, q_lo + ((c * 2 * kHalfTile + k4 * 32) >> 4), kHiK,
+                                              b_lo + ((tile * kTile + c * kHalfTile + k4 * 32) >> 4), kHiK, kIdescQK,
+                                              (c | k4) != 0);
                 tc_commit(smem_u32(&tl->s_full[sb.idx]));
                 tc_commit(smem_u32(&tl->k_empty[ks.idx]));
                 sb.advance(2);
                 ks.advance(kKStages);
-                e = next_entry(it, e, g.k_top, &cur);
+                e = next_entry(rows, e, g.k_top, &cur);
                 if (e >= g.k_top) tc_commit(smem_u32(&tl->q_empty));  // that was the pair's last use of Q
             }
             if (have_prev) {  // O = P [V_a; V_b] of the entry before
@@ -202,11 +228,11 @@ __device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned p_
                 if (!wait(smem_u32(&tl->o_empty[ob.idx]), ob.phase ^ 1, tl, 206)) return;
                 tc_fence_after();
                 const unsigned d_tmem = tmem_base + 256 + ob.idx * 128;
-                const unsigned b_base = v_smem + vs.idx * kOperand;
+                const unsigned b_lo = v_lo + vs.idx * (kOperand >> 4);
 #pragma unroll
-                for (int s = 0; s < 8; ++s)  // 16 keys per step: P column half s / 4, V rows 16 s ..
-                    tc_mma_bf16(d_tmem, smem_desc_sw128(p_smem + (s >> 2) * 2 * kHalfTile + (s & 3) * 32, 16, 1024),
-                                smem_desc_sw128(b_base + s * 2048, 2 * kHalfTile, 1024), kIdescPV, s != 0);
+                for (int s = 0; s < 8; ++s)  // 16 keys per step: P column half = V tile = s / 4
+                    tc_mma_bf16_split(d_tmem, p_lo + (((s >> 2) * 2 * kHalfTile + (s & 3) * 32) >> 4), kHiK,
+                                      b_lo + (((s >> 2) * kTile + (s & 3) * 2048) >> 4), kHiK, kIdescPV, s != 0);
                 tc_commit(smem_u32(&tl->o_full[ob.idx]));
                 tc_commit(smem_u32(&tl->v_empty[vs.idx]));
                 ob.advance(2);
@@ -214,49 +240,66 @@ __device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned p_
             }
             have_prev = have_cur;
         }
+        mbar_arrive(smem_u32(&tl->m_empty[ms.idx]));
+        ms.advance(kMaskSlots);
     }
 }
 
-// o[0..127] = o * alpha + O, O being this thread's lane of a 128-column TMEM buffer.
+// o[0..63] = o * alpha + O, O being 64 columns of this thread's lane of a TMEM buffer.
 __device__ __forceinline__ void fold_output(float *o, float alpha, unsigned taddr) {
+    unsigned r[64];
+    tmem_ld_32x32_issue(taddr, r);
+    tmem_ld_32x32_issue(taddr + 32, r + 32);
+    tmem_ld_wait();
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
-        unsigned r[32];
-        tmem_ld_32x32_issue(taddr + c * 32, r);
-        tmem_ld_wait();
-#pragma unroll
-        for (int i = 0; i < 32; ++i) o[c * 32 + i] = fmaf(o[c * 32 + i], alpha, __uint_as_float(r[i]));
-    }
+    for (int i = 0; i < 64; ++i) o[i] = fmaf(o[i], alpha, __uint_as_float(r[i]));
 }
 
+// Eight softmax warps. Warps w and w + 4 share the 32 TMEM lanes (query tokens) 32 (w % 4) ..: the
+// first takes keys 0..31 of the token's block and output channels 0..63, the second keys 32..63
+// and channels 64..127. The two exchange their partial row maxima (and, at the end, sums)
+// through shared memory, meeting on an mbarrier of their own.
 __device__ void softmax_role(const Params &P, Tail *tl, unsigned char *p_ptr, unsigned tmem_base, int t) {
     const Geom &g = P.g;
-    const int lane = t & 31, half = t >> 6, mq = t & 63;
-    const unsigned lane_off = (unsigned)(t & ~31) << 16;
+    const int lane = t & 31, row = t & 127, part = t >> 7, half = row >> 6, mq = row & 63, wq = row >> 5;
+    const unsigned lane_off = (unsigned)(row & ~31) << 16;
     // this thread's row of the block-diagonal P operand: column half = its row of the pair
-    unsigned char *p_row = p_ptr + half * 2 * kHalfTile + (t >> 3) * 1024 + (t & 7) * 128;
-    const int sw = t & 7;
-    Ring sb, ob;
+    unsigned char *p_row = p_ptr + half * 2 * kHalfTile + (row >> 3) * 1024 + (row & 7) * 128;
+    const int sw = row & 7;
+    const unsigned x_bar = smem_u32(&tl->x_bar[wq]);
+    unsigned x_par = 0;
+    int x_buf = 0;
+    // publish v, meet the partner warp, return the partner's value
+    auto exchange = [&](float v, float *other) -> bool {
+        tl->xch[x_buf][row][part] = v;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(x_bar);
+        if (!wait(x_bar, x_par, tl, 304)) return false;
+        x_par ^= 1;
+        *other = tl->xch[x_buf][row][part ^ 1];
+        x_buf ^= 1;
+        return true;
+    };
+    Ring sb, ob, ms;
     for (int id = blockIdx.x; id < P.n_items; id += gridDim.x) {
         const Item it = decode_item(P, id);
         const long long tq = (long long)it.qb * kBlk + mq;
         const bool row_active = half < it.R && tq < g.T;
-        float o[kD];
+        if (!wait(smem_u32(&tl->m_full[ms.idx]), ms.phase, tl, 305)) return;
+        const int *rows = tl->rows[ms.idx][0];
+        float o[64];
 #pragma unroll
-        for (int i = 0; i < kD; ++i) o[i] = 0.f;
+        for (int i = 0; i < 64; ++i) o[i] = 0.f;
         float m = -CUDART_INF_F, l = 0.f, alpha_prev = 1.f;
         bool have_prev = false;
         Entry cur;
-        int e = next_entry(it, -1, g.k_top, &cur);
+        int e = next_entry(rows, -1, g.k_top, &cur);
         while (e < g.k_top) {
-            // logits of this token against its row's key block
+            // this token's logits against keys 32 part .. 32 part + 31 of its row's key block
             if (!wait(smem_u32(&tl->s_full[sb.idx]), sb.phase, tl, 301)) return;
             tc_fence_after();
-            unsigned r[64];
-            const unsigned s_addr = tmem_base + sb.idx * 128 + half * 64 + lane_off;
-            tmem_ld_32x32_issue(s_addr, r);
-            tmem_ld_32x32_issue(s_addr + 32, r + 32);
-            tmem_ld_wait();
+            float sv[32];
+            tmem_ld_32x32(tmem_base + sb.idx * 128 + half * 64 + part * 32 + lane_off, sv);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&tl->s_empty[sb.idx]));
@@ -270,31 +313,35 @@ __device__ void softmax_role(const Params &P, Tail *tl, unsigned char *p_ptr, un
                 if (g.causal) lim = min(lim, tq - k0 + 1);
                 n_hi = (int)max(0ll, min(lim, (long long)kBlk));
             }
-            float mx = -CUDART_INF_F;
-            if (n_hi == kBlk) {
+            n_hi -= part * 32;  // in this thread's 32 keys
+            float mx4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
+            if (n_hi >= 32) {
 #pragma unroll
-                for (int i = 0; i < 64; ++i) mx = fmaxf(mx, __uint_as_float(r[i]));
+                for (int i = 0; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], sv[i]);
             } else {
 #pragma unroll
-                for (int i = 0; i < 64; ++i) mx = fmaxf(mx, i < n_hi ? __uint_as_float(r[i]) : -CUDART_INF_F);
+                for (int i = 0; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], i < n_hi ? sv[i] : -CUDART_INF_F);
             }
-            const float m_new = fmaxf(m, mx);
+            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+            float mx_other;
+            if (!exchange(mx, &mx_other)) return;
+            const float m_new = fmaxf(m, fmaxf(mx, mx_other));
             // with no key allowed so far m_new is -inf: every p is 0 and nothing is rescaled
             const float shift = m_new == -CUDART_INF_F ? 0.f : -m_new * P.scale_log2;
             const float alpha = m_new == m ? 1.f : exp2f((m - m_new) * P.scale_log2);
-            float sum = 0.f;
-            unsigned packed[32];
+            float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+            unsigned packed[16];
 #pragma unroll
-            for (int i = 0; i < 64; i += 2) {
-                float p0 = exp2f(fmaf(__uint_as_float(r[i]), P.scale_log2, shift));
-                float p1 = exp2f(fmaf(__uint_as_float(r[i + 1]), P.scale_log2, shift));
+            for (int i = 0; i < 32; i += 2) {
+                float p0 = exp2f(fmaf(sv[i], P.scale_log2, shift));
+                float p1 = exp2f(fmaf(sv[i + 1], P.scale_log2, shift));
                 p0 = i < n_hi ? p0 : 0.f;
                 p1 = i + 1 < n_hi ? p1 : 0.f;
-                sum += p0 + p1;
+                sum4[(i >> 1) & 3] += p0 + p1;
                 __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
                 packed[i >> 1] = *reinterpret_cast<unsigned *>(&pk);
             }
-            l = l * alpha + sum;
+            l = l * alpha + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
             m = m_new;
             // the P buffer is free, and the previous product ready, once the previous P V chain is done
             if (have_prev) {
@@ -302,14 +349,14 @@ __device__ void softmax_role(const Params &P, Tail *tl, unsigned char *p_ptr, un
                 tc_fence_after();
             }
 #pragma unroll
-            for (int c = 0; c < 8; ++c)
-                *reinterpret_cast<uint4 *>(p_row + ((c ^ sw) << 4)) =
+            for (int c = 0; c < 4; ++c)
+                *reinterpret_cast<uint4 *>(p_row + (((part * 4 + c) ^ sw) << 4)) =
                     make_uint4(packed[4 * c], packed[4 * c + 1], packed[4 * c + 2], packed[4 * c + 3]);
             fence_async_smem();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&tl->p_full));
             if (have_prev) {
-                fold_output(o, alpha_prev, tmem_base + 256 + ob.idx * 128 + lane_off);
+                fold_output(o, alpha_prev, tmem_base + 256 + ob.idx * 128 + part * 64 + lane_off);
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&tl->o_empty[ob.idx]));
@@ -317,22 +364,28 @@ __device__ void softmax_role(const Params &P, Tail *tl, unsigned char *p_ptr, un
             }
             alpha_prev = alpha;
             have_prev = true;
-            e = next_entry(it, e, g.k_top, &cur);
+            e = next_entry(rows, e, g.k_top, &cur);
         }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&tl->m_empty[ms.idx]));
+        ms.advance(kMaskSlots);
         if (have_prev) {
             if (!wait(smem_u32(&tl->o_full[ob.idx]), ob.phase, tl, 303)) return;
             tc_fence_after();
-            fold_output(o, alpha_prev, tmem_base + 256 + ob.idx * 128 + lane_off);
+            fold_output(o, alpha_prev, tmem_base + 256 + ob.idx * 128 + part * 64 + lane_off);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&tl->o_empty[ob.idx]));
             ob.advance(2);
         }
+        float l_other;
+        if (!exchange(l, &l_other)) return;
         if (row_active) {
-            const float inv = l > 0.f ? 1.f / l : 0.f;
-            uint4 *dst = reinterpret_cast<uint4 *>(P.out + (((long long)it.b * g.H + it.h0 + half) * g.T + tq) * kD);
+            const float lt = l + l_other;
+            const float inv = lt > 0.f ? 1.f / lt : 0.f;
+            uint4 *dst = reinterpret_cast<uint4 *>(P.out + (((long long)it.b * g.H + it.h0 + half) * g.T + tq) * kD + part * 64);
 #pragma unroll
-            for (int c = 0; c < 16; ++c) {
+            for (int c = 0; c < 8; ++c) {
                 unsigned w[4];
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
@@ -361,10 +414,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         for (int i = 0; i < kKStages; ++i) { mbar_init(smem_u32(&tl->k_full[i]), 1); mbar_init(smem_u32(&tl->k_empty[i]), 1); }
         for (int i = 0; i < kVStages; ++i) { mbar_init(smem_u32(&tl->v_full[i]), 1); mbar_init(smem_u32(&tl->v_empty[i]), 1); }
         for (int i = 0; i < 2; ++i) {
-            mbar_init(smem_u32(&tl->s_full[i]), 1); mbar_init(smem_u32(&tl->s_empty[i]), 4);
-            mbar_init(smem_u32(&tl->o_full[i]), 1); mbar_init(smem_u32(&tl->o_empty[i]), 4);
+            mbar_init(smem_u32(&tl->s_full[i]), 1); mbar_init(smem_u32(&tl->s_empty[i]), 8);
+            mbar_init(smem_u32(&tl->o_full[i]), 1); mbar_init(smem_u32(&tl->o_empty[i]), 8);
         }
-        mbar_init(smem_u32(&tl->p_full), 4);
+        mbar_init(smem_u32(&tl->p_full), 8);
+        for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&tl->x_bar[i]), 2);
+        for (int i = 0; i < kMaskSlots; ++i) { mbar_init(smem_u32(&tl->m_full[i]), 1); mbar_init(smem_u32(&tl->m_empty[i]), 10); }
         tl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -382,6 +437,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         if (lane == 0) producer_role(P, &tmap_q, &tmap_k, &tmap_v, tl, q_smem, k_smem, v_smem);
     } else if (warp == 1) {
         if (lane == 0) mma_role(P, tl, q_smem, p_smem, k_smem, v_smem, tmem_base);
+    } else if (warp == 2) {
+        mask_loader_role(P, tl, lane);
     } else if (warp >= 4) {
         softmax_role(P, tl, smem + kOperand, tmem_base, (int)threadIdx.x - 128);
     }
@@ -404,7 +461,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
 }  // namespace
 
 bool attn_tc_supported(const Geom &g, int dtype) {
-    return dtype == STREAM_BF16 && g.d == kD && g.bq == kBlk && g.bk == kBlk && tma_strides_ok(g);
+    return dtype == STREAM_BF16 && g.d == kD && g.bq == kBlk && g.bk == kBlk && g.k_top <= kMaxKTopTc && tma_strides_ok(g);
 }
 
 stream_status launch_attn_tc(const Geom &g, const void *q, const void *k, const void *v, const int32_t *mask,
@@ -414,11 +471,11 @@ stream_status launch_attn_tc(const Geom &g, const void *q, const void *k, const 
         return STREAM_ERR_UNSUPPORTED;
     }
     CUtensorMap tq, tk, tv;
-    stream_status rc = make_map_bf16_d128(&tq, q, g.T, g.H, g.batch, g.qs_t, g.qs_h, g.qs_b, "q");
+    stream_status rc = make_map5_bf16_d128(&tq, q, g.T, g.H, g.batch, g.qs_t, g.qs_h, g.qs_b, 2, "q");
     if (rc != STREAM_OK) return rc;
-    rc = make_map_bf16_d128(&tk, k, g.T, g.G, g.batch, g.ks_t, g.ks_h, g.ks_b, "k");
+    rc = make_map5_bf16_d128(&tk, k, g.T, g.G, g.batch, g.ks_t, g.ks_h, g.ks_b, 1, "k");
     if (rc != STREAM_OK) return rc;
-    rc = make_map_bf16_d128(&tv, v, g.T, g.G, g.batch, g.ks_t, g.ks_h, g.ks_b, "v");
+    rc = make_map5_bf16_d128(&tv, v, g.T, g.G, g.batch, g.ks_t, g.ks_h, g.ks_b, 1, "v");
     if (rc != STREAM_OK) return rc;
     Params P;
     P.g = g;

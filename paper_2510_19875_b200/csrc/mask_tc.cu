@@ -54,8 +54,8 @@ __device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, Tail *t
     return mbar_wait_bounded(bar, parity, &tl->abort_flag, &ws->error, &ws->error_info, code);
 }
 
-// K-major, 128-byte-swizzled operand with 8-row groups 1024 bytes apart.
-__device__ __forceinline__ unsigned long long smem_desc(unsigned addr) { return smem_desc_sw128(addr, 16, 1024); }
+// K-major, 128-byte-swizzled operands with 8-row groups 1024 bytes apart: high descriptor word.
+constexpr unsigned kDescHi = desc_hi_sw128(1024);
 
 // D fp32, A and B bf16, both K-major, M = 128, N = 64.
 constexpr unsigned kIdesc = idesc_bf16(128, 64, false);
@@ -117,6 +117,7 @@ __device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_
     const Geom &g = P.g;
     Ring st, sl;
     unsigned grp_par = 0, q_par = 0, jr_par[kR] = {0, 0, 0, 0};
+    const unsigned q_lo = desc_lo_sw128(q_smem, 16);
     for (;;) {
         if (!mbar_wait(smem_u32(&tl->jobs_ready[kR]), grp_par, tl, P.ws, 201)) return;
         grp_par ^= 1;
@@ -135,18 +136,19 @@ __device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_
                 const int n = tl->n_jobs[li];
                 for (int j = 0; j < n; j += 2) {
                     if (!mbar_wait(smem_u32(&tl->full[st.idx]), st.phase, tl, P.ws, 204)) return;
-                    const unsigned a_base = k_smem + st.idx * kStageBytes;
+                    const unsigned a_lo = desc_lo_sw128(k_smem + st.idx * kStageBytes, 16);
                     const int r0 = level == 0 ? 0 : x, r1 = level == 0 ? R : x + 1;
                     for (int r = r0; r < r1; ++r) {
                         if (!mbar_wait(smem_u32(&tl->tmem_empty[sl.idx]), sl.phase ^ 1, tl, P.ws, 205)) return;
                         tc_fence_after();
                         const unsigned d_tmem = tmem_base + sl.idx * 64;
+                        const unsigned b_lo = q_lo + r * (kHalfTile >> 4);
 #pragma unroll
                         for (int c = 0; c < 2; ++c)
 #pragma unroll
                             for (int k4 = 0; k4 < 4; ++k4)
-                                tc_mma_bf16(d_tmem, smem_desc(a_base + c * 2 * kHalfTile + k4 * 32),
-                                            smem_desc(q_smem + (c * kR + r) * kHalfTile + k4 * 32), kIdesc, (c | k4) != 0);
+                                tc_mma_bf16_split(d_tmem, a_lo + ((c * 2 * kHalfTile + k4 * 32) >> 4), kDescHi,
+                                                  b_lo + ((c * kR * kHalfTile + k4 * 32) >> 4), kDescHi, kIdesc, (c | k4) != 0);
                         tc_commit(smem_u32(&tl->tmem_full[sl.idx]));
                         sl.advance(kSlots);
                     }

@@ -33,9 +33,8 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
 // Bounded wait on an mbarrier phase. Returns false if the CTA is aborting, or if this wait ran
 // out, in which case it raises the CTA's abort flag and records `code` (first one wins) with the
 // block index in the two error words.
-static __device__ __noinline__ bool mbar_wait_bounded(unsigned bar, unsigned parity, int *abort_flag, unsigned *err_code,
-                                               unsigned *err_info, unsigned code) {
-    if (mbar_try_wait(bar, parity)) return true;
+static __device__ __noinline__ bool mbar_wait_slow(unsigned bar, unsigned parity, int *abort_flag, unsigned *err_code,
+                                                   unsigned *err_info, unsigned code) {
     const long long t0 = clock64();
     for (;;) {
         if (mbar_try_wait(bar, parity)) return true;
@@ -47,12 +46,25 @@ static __device__ __noinline__ bool mbar_wait_bounded(unsigned bar, unsigned par
         }
     }
 }
+__device__ __forceinline__ bool mbar_wait_bounded(unsigned bar, unsigned parity, int *abort_flag, unsigned *err_code,
+                                                  unsigned *err_info, unsigned code) {
+    if (mbar_try_wait(bar, parity)) return true;  // the common case costs one instruction
+    return mbar_wait_slow(bar, parity, abort_flag, err_code, err_info, code);
+}
 
 __device__ __forceinline__ void tma_load_4d(unsigned dst, const CUtensorMap *map, unsigned bar, int c0, int c1, int c2,
                                             int c3) {
     asm volatile(
         "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
         ::"r"(dst), "l"((unsigned long long)map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+
+__device__ __forceinline__ void tma_load_5d(unsigned dst, const CUtensorMap *map, unsigned bar, int c0, int c1, int c2,
+                                            int c3, int c4) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+        ::"r"(dst), "l"((unsigned long long)map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
         : "memory");
 }
 
@@ -70,6 +82,18 @@ __device__ __forceinline__ void tc_mma_bf16(unsigned d_tmem, unsigned long long 
     asm volatile(
         "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// The same with both descriptors given as (low word, high word). The low word holds the start
+// address in 16-byte units, so a K step is one 32-bit add on it; the high word never changes
+// for a given operand layout.
+__device__ __forceinline__ void tc_mma_bf16_split(unsigned d_tmem, unsigned a_lo, unsigned a_hi, unsigned b_lo,
+                                                  unsigned b_hi, unsigned idesc, unsigned accumulate) {
+    asm volatile(
+        "{\n.reg .pred p;\n.reg .b64 da, db;\nmov.b64 da, {%1, %2};\nmov.b64 db, {%3, %4};\nsetp.ne.b32 p, %6, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
         : "memory");
 }
 
@@ -120,6 +144,12 @@ __device__ __forceinline__ unsigned long long smem_desc_sw128(unsigned addr, uns
            ((unsigned long long)((sbo >> 4) & 0x3FFF) << 32) | (1ull << 46) | (2ull << 61);
 }
 
+// Low and high words of that descriptor; (addr_bytes >> 4) is added to the low word per operand.
+__device__ __forceinline__ unsigned desc_lo_sw128(unsigned addr, unsigned lbo) {
+    return ((addr >> 4) & 0x3FFF) | (((lbo >> 4) & 0x3FFF) << 16);
+}
+constexpr unsigned desc_hi_sw128(unsigned sbo) { return ((sbo >> 4) & 0x3FFF) | (1u << 14) | (2u << 29); }
+
 // kind::f16 instruction descriptor: D fp32, A and B bf16, A K-major, B K-major or MN-major.
 constexpr unsigned idesc_bf16(unsigned M, unsigned N, bool b_mn_major) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((N >> 3) << 17) | ((M >> 4) << 24);
@@ -165,6 +195,27 @@ inline stream_status make_map_bf16_d128(CUtensorMap *map, const void *base, long
     cuuint64_t strides[3] = {(cuuint64_t)s_t * 2, (cuuint64_t)s_h * 2, (cuuint64_t)s_b * 2};
     cuuint32_t box[4] = {64, 64, 1, 1}, estr[4] = {1, 1, 1, 1};
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled(%s) failed with %d", what, (int)r); return STREAM_ERR_CUDA; }
+    return STREAM_OK;
+}
+
+// The same tensor seen as [batch, heads, 2 channel halves, T, 64]: one box brings a whole
+// 64-token x 128-channel tile (16 KB) as [half][64 rows][128 B], the layout of a 128-byte-swizzled
+// K-major (or, read along the rows, MN-major) tcgen05 operand. With heads_in_box = 2 the two
+// heads h, h + 1 land as [half][head][64 rows][128 B]: a 128-row operand per half.
+// Coordinates: (0, token, head, 0, batch) with the half as dimension 3.
+inline stream_status make_map5_bf16_d128(CUtensorMap *map, const void *base, long long T, int heads, int batch,
+                                         long long s_t, long long s_h, long long s_b, int heads_in_box, const char *what) {
+    EncodeTiledFn fn = encode_fn();
+    if (fn == nullptr) { set_error("cuTensorMapEncodeTiled is not available from this driver"); return STREAM_ERR_CUDA; }
+    if (heads == 1) s_h = s_t * T;
+    if (batch == 1) s_b = s_h * heads;
+    cuuint64_t dims[5] = {64, (cuuint64_t)T, (cuuint64_t)heads, 2, (cuuint64_t)batch};
+    cuuint64_t strides[4] = {(cuuint64_t)s_t * 2, (cuuint64_t)s_h * 2, 128, (cuuint64_t)s_b * 2};
+    cuuint32_t box[5] = {64, 64, (cuuint32_t)heads_in_box, 2, 1}, estr[5] = {1, 1, 1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void *>(base), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) { set_error("cuTensorMapEncodeTiled(%s) failed with %d", what, (int)r); return STREAM_ERR_CUDA; }

@@ -75,6 +75,11 @@ __device__ __forceinline__ bool wait(unsigned bar, unsigned parity, Tail *tl, un
     return mbar_wait_bounded(bar, parity, &tl->abort_flag, &g_attn_status[0], &g_attn_status[1], code);
 }
 
+// The same for a whole converged warp (all lanes get the same answer).
+__device__ __forceinline__ bool wait_w(unsigned bar, unsigned parity, Tail *tl, unsigned code) {
+    return mbar_wait_warp(bar, parity, &tl->abort_flag, &g_attn_status[0], &g_attn_status[1], code);
+}
+
 // The pair a CTA works on in its n-th round.
 struct Item {
     int b, kvh, qb, h0, R;
@@ -178,6 +183,7 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
     }
 }
 
+// Run by all 32 lanes of its warp, converged: the waits are warp-wide, one elected lane issues.
 __device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned p_smem, unsigned k_smem, unsigned v_smem,
                          unsigned tmem_base) {
     const Geom &g = P.g;
@@ -188,59 +194,66 @@ __device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned p_
     const unsigned q_lo = desc_lo_sw128(q_smem, 16), p_lo = desc_lo_sw128(p_smem, 16), k_lo = desc_lo_sw128(k_smem, 16),
                    v_lo = desc_lo_sw128(v_smem, kHalfTile);
     for (int id = blockIdx.x; id < P.n_items; id += gridDim.x) {
-        if (!wait(smem_u32(&tl->m_full[ms.idx]), ms.phase, tl, 207)) return;
+        if (!wait_w(smem_u32(&tl->m_full[ms.idx]), ms.phase, tl, 207)) return;
         const int *rows = tl->rows[ms.idx][0];
         Entry cur;
         int e = next_entry(rows, -1, g.k_top, &cur);
         if (e < g.k_top) {
-            if (!wait(smem_u32(&tl->q_full), q_par, tl, 201)) return;
+            if (!wait_w(smem_u32(&tl->q_full), q_par, tl, 201)) return;
             q_par ^= 1;
         }
         bool have_prev = false;
         while (e < g.k_top || have_prev) {
             const bool have_cur = e < g.k_top;
             if (have_cur) {  // S = [Q_0; Q_1] [K_a; K_b]^T, one chain per K tile
-                if (!wait(smem_u32(&tl->k_full[ks.idx]), ks.phase, tl, 202)) return;
-                if (!wait(smem_u32(&tl->s_empty[sb.idx]), sb.phase ^ 1, tl, 203)) return;
+                if (!wait_w(smem_u32(&tl->k_full[ks.idx]), ks.phase, tl, 202)) return;
+                if (!wait_w(smem_u32(&tl->s_empty[sb.idx]), sb.phase ^ 1, tl, 203)) return;
                 tc_fence_after();
                 const unsigned d_tmem = tmem_base + sb.idx * 128;
                 const unsigned b_lo = k_lo + ks.idx * (kOperand >> 4);
+                e = next_entry(rows, e, g.k_top, &cur);
+                if (elect_one()) {
 #pragma unroll
-                for (int tile = 0; tile < 2; ++tile)
+                    for (int tile = 0; tile < 2; ++tile)
 #pragma unroll
-                    for (int c = 0; c < 2; ++c)
+                        for (int c = 0; c < 2; ++c)
 #pragma unroll
-                        for (int k4 = 0; k4 < 4; ++k4)
-                            tc_mma_bf16_split(d_tmem + tile * 64, q_lo + ((c * 2 * kHalfTile + k4 * 32) >> 4), kHiK,
-                                              b_lo + ((tile * kTile + c * kHalfTile + k4 * 32) >> 4), kHiK, kIdescQK,
-                                              (c | k4) != 0);
-                tc_commit(smem_u32(&tl->s_full[sb.idx]));
-                tc_commit(smem_u32(&tl->k_empty[ks.idx]));
+                            for (int k4 = 0; k4 < 4; ++k4)
+                                tc_mma_bf16_split(d_tmem + tile * 64, q_lo + ((c * 2 * kHalfTile + k4 * 32) >> 4), kHiK,
+                                                  b_lo + ((tile * kTile + c * kHalfTile + k4 * 32) >> 4), kHiK, kIdescQK,
+                                                  (c | k4) != 0);
+                    tc_commit(smem_u32(&tl->s_full[sb.idx]));
+                    tc_commit(smem_u32(&tl->k_empty[ks.idx]));
+                    if (e >= g.k_top) tc_commit(smem_u32(&tl->q_empty));  // that was the pair's last use of Q
+                }
+                __syncwarp();
                 sb.advance(2);
                 ks.advance(kKStages);
-                e = next_entry(rows, e, g.k_top, &cur);
-                if (e >= g.k_top) tc_commit(smem_u32(&tl->q_empty));  // that was the pair's last use of Q
             }
             if (have_prev) {  // O = P [V_a; V_b] of the entry before
-                if (!wait(smem_u32(&tl->p_full), p_par, tl, 204)) return;
+                if (!wait_w(smem_u32(&tl->p_full), p_par, tl, 204)) return;
                 p_par ^= 1;
-                if (!wait(smem_u32(&tl->v_full[vs.idx]), vs.phase, tl, 205)) return;
-                if (!wait(smem_u32(&tl->o_empty[ob.idx]), ob.phase ^ 1, tl, 206)) return;
+                if (!wait_w(smem_u32(&tl->v_full[vs.idx]), vs.phase, tl, 205)) return;
+                if (!wait_w(smem_u32(&tl->o_empty[ob.idx]), ob.phase ^ 1, tl, 206)) return;
                 tc_fence_after();
                 const unsigned d_tmem = tmem_base + 256 + ob.idx * 128;
                 const unsigned b_lo = v_lo + vs.idx * (kOperand >> 4);
+                if (elect_one()) {
 #pragma unroll
-                for (int s = 0; s < 8; ++s)  // 16 keys per step: P column half = V tile = s / 4
-                    tc_mma_bf16_split(d_tmem, p_lo + (((s >> 2) * 2 * kHalfTile + (s & 3) * 32) >> 4), kHiK,
-                                      b_lo + (((s >> 2) * kTile + (s & 3) * 2048) >> 4), kHiK, kIdescPV, s != 0);
-                tc_commit(smem_u32(&tl->o_full[ob.idx]));
-                tc_commit(smem_u32(&tl->v_empty[vs.idx]));
+                    for (int s = 0; s < 8; ++s)  // 16 keys per step: P column half = V tile = s / 4
+                        tc_mma_bf16_split(d_tmem, p_lo + (((s >> 2) * 2 * kHalfTile + (s & 3) * 32) >> 4), kHiK,
+                                          b_lo + (((s >> 2) * kTile + (s & 3) * 2048) >> 4), kHiK, kIdescPV, s != 0);
+                    tc_commit(smem_u32(&tl->o_full[ob.idx]));
+                    tc_commit(smem_u32(&tl->v_empty[vs.idx]));
+                }
+                __syncwarp();
                 ob.advance(2);
                 vs.advance(kVStages);
             }
             have_prev = have_cur;
         }
-        mbar_arrive(smem_u32(&tl->m_empty[ms.idx]));
+        if (elect_one()) mbar_arrive(smem_u32(&tl->m_empty[ms.idx]));
+        __syncwarp();
         ms.advance(kMaskSlots);
     }
 }
@@ -436,7 +449,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     if (warp == 0) {
         if (lane == 0) producer_role(P, &tmap_q, &tmap_k, &tmap_v, tl, q_smem, k_smem, v_smem);
     } else if (warp == 1) {
-        if (lane == 0) mma_role(P, tl, q_smem, p_smem, k_smem, v_smem, tmem_base);
+        mma_role(P, tl, q_smem, p_smem, k_smem, v_smem, tmem_base);
     } else if (warp == 2) {
         mask_loader_role(P, tl, lane);
     } else if (warp >= 4) {

@@ -54,6 +54,11 @@ __device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, Tail *t
     return mbar_wait_bounded(bar, parity, &tl->abort_flag, &ws->error, &ws->error_info, code);
 }
 
+// The same for a whole converged warp (all lanes get the same answer).
+__device__ __forceinline__ bool mbar_wait_w(unsigned bar, unsigned parity, Tail *tl, WorkspaceHeader *ws, unsigned code) {
+    return mbar_wait_warp(bar, parity, &tl->abort_flag, &ws->error, &ws->error_info, code);
+}
+
 // K-major, 128-byte-swizzled operands with 8-row groups 1024 bytes apart: high descriptor word.
 constexpr unsigned kDescHi = desc_hi_sw128(1024);
 
@@ -113,46 +118,50 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
     }
 }
 
+// Run by all 32 lanes of its warp, converged: the waits are warp-wide, one elected lane issues.
 __device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_smem, unsigned tmem_base) {
     const Geom &g = P.g;
     Ring st, sl;
     unsigned grp_par = 0, q_par = 0, jr_par[kR] = {0, 0, 0, 0};
     const unsigned q_lo = desc_lo_sw128(q_smem, 16);
     for (;;) {
-        if (!mbar_wait(smem_u32(&tl->jobs_ready[kR]), grp_par, tl, P.ws, 201)) return;
+        if (!mbar_wait_w(smem_u32(&tl->jobs_ready[kR]), grp_par, tl, P.ws, 201)) return;
         grp_par ^= 1;
         if (tl->grp_id < 0) return;
         const int R = tl->grp_R;
-        if (!mbar_wait(smem_u32(&tl->q_full), q_par, tl, P.ws, 202)) return;
+        if (!mbar_wait_w(smem_u32(&tl->q_full), q_par, tl, P.ws, 202)) return;
         q_par ^= 1;
         for (int level = 0; level < g.levels; ++level) {
             const int lists = level == 0 ? 1 : R;
             for (int x = 0; x < lists; ++x) {
                 const int li = level == 0 ? kR : x;
                 if (level > 0) {
-                    if (!mbar_wait(smem_u32(&tl->jobs_ready[x]), jr_par[x], tl, P.ws, 203)) return;
+                    if (!mbar_wait_w(smem_u32(&tl->jobs_ready[x]), jr_par[x], tl, P.ws, 203)) return;
                     jr_par[x] ^= 1;
                 }
                 const int n = tl->n_jobs[li];
                 for (int j = 0; j < n; j += 2) {
-                    if (!mbar_wait(smem_u32(&tl->full[st.idx]), st.phase, tl, P.ws, 204)) return;
+                    if (!mbar_wait_w(smem_u32(&tl->full[st.idx]), st.phase, tl, P.ws, 204)) return;
                     const unsigned a_lo = desc_lo_sw128(k_smem + st.idx * kStageBytes, 16);
                     const int r0 = level == 0 ? 0 : x, r1 = level == 0 ? R : x + 1;
                     for (int r = r0; r < r1; ++r) {
-                        if (!mbar_wait(smem_u32(&tl->tmem_empty[sl.idx]), sl.phase ^ 1, tl, P.ws, 205)) return;
+                        if (!mbar_wait_w(smem_u32(&tl->tmem_empty[sl.idx]), sl.phase ^ 1, tl, P.ws, 205)) return;
                         tc_fence_after();
                         const unsigned d_tmem = tmem_base + sl.idx * 64;
                         const unsigned b_lo = q_lo + r * (kHalfTile >> 4);
+                        if (elect_one()) {
 #pragma unroll
-                        for (int c = 0; c < 2; ++c)
+                            for (int c = 0; c < 2; ++c)
 #pragma unroll
-                            for (int k4 = 0; k4 < 4; ++k4)
-                                tc_mma_bf16_split(d_tmem, a_lo + ((c * 2 * kHalfTile + k4 * 32) >> 4), kDescHi,
-                                                  b_lo + ((c * kR * kHalfTile + k4 * 32) >> 4), kDescHi, kIdesc, (c | k4) != 0);
-                        tc_commit(smem_u32(&tl->tmem_full[sl.idx]));
+                                for (int k4 = 0; k4 < 4; ++k4)
+                                    tc_mma_bf16_split(d_tmem, a_lo + ((c * 2 * kHalfTile + k4 * 32) >> 4), kDescHi,
+                                                      b_lo + ((c * kR * kHalfTile + k4 * 32) >> 4), kDescHi, kIdesc, (c | k4) != 0);
+                            tc_commit(smem_u32(&tl->tmem_full[sl.idx]));
+                            if (r + 1 == r1) tc_commit(smem_u32(&tl->empty[st.idx]));
+                        }
+                        __syncwarp();
                         sl.advance(kSlots);
                     }
-                    tc_commit(smem_u32(&tl->empty[st.idx]));
                     st.advance(kStages);
                 }
             }
@@ -377,7 +386,7 @@ mask_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     if (warp == 0) {
         if (lane == 0) producer_role(P, &tmap_q, &tmap_k, tl, q_smem, k_smem);
     } else if (warp == 1) {
-        if (lane == 0) mma_role(P, tl, q_smem, k_smem, tmem_base);
+        mma_role(P, tl, q_smem, k_smem, tmem_base);
     } else if (warp == 2) {
         controller_role(P, tl, lane);
     } else if (warp >= 4) {

@@ -52,6 +52,22 @@ __device__ __forceinline__ bool mbar_wait_bounded(unsigned bar, unsigned parity,
     return mbar_wait_slow(bar, parity, abort_flag, err_code, err_info, code);
 }
 
+// True in exactly one lane of a converged warp (the same lane every time).
+__device__ __forceinline__ bool elect_one() {
+    unsigned pred;
+    asm volatile("{\n.reg .pred p;\nelect.sync _|p, 0xffffffff;\nselp.u32 %0, 1, 0, p;\n}" : "=r"(pred));
+    return pred != 0;
+}
+
+// mbar_wait_bounded for a whole converged warp: every lane waits, and all lanes get the same
+// answer (false as soon as one lane saw the abort flag or ran out of time), so that the warp
+// stays converged for the elect_one() that follows.
+__device__ __forceinline__ bool mbar_wait_warp(unsigned bar, unsigned parity, int *abort_flag, unsigned *err_code,
+                                               unsigned *err_info, unsigned code) {
+    const bool ok = mbar_wait_bounded(bar, parity, abort_flag, err_code, err_info, code);
+    return __all_sync(0xffffffffu, ok);
+}
+
 __device__ __forceinline__ void tma_load_4d(unsigned dst, const CUtensorMap *map, unsigned bar, int c0, int c1, int c2,
                                             int c3) {
     asm volatile(
@@ -148,10 +164,10 @@ __device__ __forceinline__ unsigned long long smem_desc_sw128(unsigned addr, uns
 __device__ __forceinline__ unsigned desc_lo_sw128(unsigned addr, unsigned lbo) {
     return ((addr >> 4) & 0x3FFF) | (((lbo >> 4) & 0x3FFF) << 16);
 }
-constexpr unsigned desc_hi_sw128(unsigned sbo) { return ((sbo >> 4) & 0x3FFF) | (1u << 14) | (2u << 29); }
+__host__ __device__ constexpr unsigned desc_hi_sw128(unsigned sbo) { return ((sbo >> 4) & 0x3FFF) | (1u << 14) | (2u << 29); }
 
 // kind::f16 instruction descriptor: D fp32, A and B bf16, A K-major, B K-major or MN-major.
-constexpr unsigned idesc_bf16(unsigned M, unsigned N, bool b_mn_major) {
+__host__ __device__ constexpr unsigned idesc_bf16(unsigned M, unsigned N, bool b_mn_major) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((N >> 3) << 17) | ((M >> 4) << 24);
 }
 

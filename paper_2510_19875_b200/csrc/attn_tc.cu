@@ -3,9 +3,9 @@
 //
 // One persistent CTA per SM works through "pairs": two query heads of one kv head at one query
 // block. Their Q tiles are stacked into one 128-row A operand. For every mask entry e the two
-// rows name one key block each (K_a, K_b, usually different); each tile arrives by one TMA box
-// (128-byte swizzle) and
-//     S = [Q_0; Q_1] [K_a; K_b]^T      (128 x 128, fp32 in TMEM; one N = 64 chain per tile)
+// rows name one key block each (K_a, K_b, usually different); the tiles arrive by TMA (128-byte
+// swizzle), stacked too, and
+//     S = [Q_0; Q_1] [K_a; K_b]^T      (128 x 128, fp32 in TMEM)
 // holds row 0's logits in its upper-left quadrant and row 1's in its lower-right one. The
 // softmax warps own one TMEM lane (= one query token) per thread pair: they read its 64 logits,
 // apply the element-level mask C, update the running maximum and sum (online softmax, fp32), and
@@ -16,12 +16,15 @@
 // output registers (o = o * alpha + O_e) one iteration later, so that the tensor core works on
 // the next logits meanwhile.
 //
-// Roles (384 threads): warp 0 TMA producer, warp 1 MMA issuer + TMEM owner, warp 2 copies the
-// pairs' mask rows from global to shared memory ahead of everyone else, warps 4..11 softmax (two
-// threads per query token: half of its keys and half of its output channels each). Every role
-// walks the same sequence of (pair, entry), read from the shared copy of the mask rows; they meet
-// only on mbarriers. Every wait is bounded: on a timeout the CTA records a code in a device status
-// word, raises a shared abort flag, lets its copies drain and leaves.
+// Roles (384 threads): warp 0 TMA producer; warp 1 issues the Q K^T chains and owns TMEM; warp 3
+// issues the P V chains (two issuing warps, because the thread that issues a chain is held until
+// the tensor core has taken it: with one warp the waits and commits between chains would not
+// overlap with the chains themselves); warp 2 copies the pairs' mask rows from global to shared
+// memory ahead of everyone else; warps 4..11 softmax (two threads per query token: half of its
+// keys and half of its output channels each). Every role walks the same sequence of (pair,
+// entry), read from the shared copy of the mask rows; they meet only on mbarriers. Every wait is
+// bounded: on a timeout the CTA records a code in a device status word, raises a shared abort
+// flag, lets its copies drain and leaves.
 #include <math_constants.h>
 
 #include "tc_common.cuh"
@@ -39,16 +42,20 @@ using namespace tc;
 constexpr int kThreads = 384;
 constexpr int kBlk = 64, kD = 128;
 constexpr int kHalfTile = kBlk * 128;       // 64 rows x 128 bytes
-constexpr int kTile = 2 * kHalfTile;        // one 64 x 128 tile as [2 channel halves][64 rows][128 B]
+constexpr int kTile = 2 * kHalfTile;        // one 64 x 128 tile
 constexpr int kOperand = 2 * kTile;         // two tiles (K_a, K_b or V_a, V_b), or a 128-row operand
-constexpr int kKStages = 2, kVStages = 2;
+constexpr int kKStages = 2, kVStages = 2;   // = S and O buffers (see Tail)
 constexpr int kMaskSlots = 2;               // pairs whose mask rows are resident
 constexpr int kMaxKTopTc = 1024;
 
 struct Tail {
     unsigned long long q_full, q_empty;
-    unsigned long long k_full[kKStages], k_empty[kKStages], v_full[kVStages], v_empty[kVStages];
-    unsigned long long s_full[2], s_empty[2], o_full[2], o_empty[2], p_full;
+    unsigned long long k_full[kKStages], v_full[kVStages];
+    // s_full also tells the producer that K stage i is free, o_full that V stage i is: the rings
+    // of K stages and S buffers (V stages and O buffers) have the same length and move together.
+    // There is no "o_empty": P of entry j is published (p_full) after the same threads folded the
+    // product of entry j - 2, and the P V warp waits for every P before it overwrites that buffer.
+    unsigned long long s_full[2], s_empty[2], o_full[2], p_full;
     unsigned long long m_full[kMaskSlots], m_empty[kMaskSlots];
     unsigned long long x_bar[4];  // softmax warps w and w + 4 meet here
     unsigned int tmem_base;
@@ -59,7 +66,7 @@ struct Tail {
 constexpr int kSmemBytes = (2 + kKStages + kVStages) * kOperand + (int)sizeof(Tail) + 1024;
 static_assert(kSmemBytes <= 232448, "exceeds the shared memory of one CTA");
 
-constexpr unsigned kIdescQK = idesc_bf16(128, 64, false);   // B = one K tile, K-major
+constexpr unsigned kIdescQK = idesc_bf16(128, 128, false);  // B = stacked K tiles, K-major
 constexpr unsigned kIdescPV = idesc_bf16(128, 128, true);   // B = stacked V tiles, MN-major
 constexpr unsigned kHiK = desc_hi_sw128(1024);              // every operand: 8-row (8-key) groups 1024 bytes apart
 
@@ -140,12 +147,21 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
     const Geom &g = P.g;
     Ring ks, vs, ms;
     unsigned q_par = 0;
-    auto load_pair = [&](const CUtensorMap *map, unsigned dst, unsigned bar, const Item &it, Entry x) {
-        // a row without a block at this entry gets block 0; its logits are masked out entirely
+    // a row without a block at an entry gets block 0; its logits are masked out entirely
+    auto load_k_pair = [&](unsigned dst, unsigned bar, const Item &it, Entry x) {  // [half][tile][64 rows][128 B]
         const int ba = x.a >= 0 ? x.a : 0, bb = x.b >= 0 ? x.b : 0;
         mbar_arrive_expect_tx(bar, (unsigned)kOperand);
-        tma_load_5d(dst, map, bar, 0, ba * kBlk, it.kvh, 0, it.b);
-        tma_load_5d(dst + kTile, map, bar, 0, bb * kBlk, it.kvh, 0, it.b);
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+            tma_load_4d(dst + c * 2 * kHalfTile, tk, bar, c * 64, ba * kBlk, it.kvh, it.b);
+            tma_load_4d(dst + c * 2 * kHalfTile + kHalfTile, tk, bar, c * 64, bb * kBlk, it.kvh, it.b);
+        }
+    };
+    auto load_v_pair = [&](unsigned dst, unsigned bar, const Item &it, Entry x) {  // [tile][half][64 rows][128 B]
+        const int ba = x.a >= 0 ? x.a : 0, bb = x.b >= 0 ? x.b : 0;
+        mbar_arrive_expect_tx(bar, (unsigned)kOperand);
+        tma_load_5d(dst, tv, bar, 0, ba * kBlk, it.kvh, 0, it.b);
+        tma_load_5d(dst + kTile, tv, bar, 0, bb * kBlk, it.kvh, 0, it.b);
     };
     for (int id = blockIdx.x; id < P.n_items; id += gridDim.x) {
         const Item it = decode_item(P, id);
@@ -157,8 +173,9 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
         while (e < g.k_top || have_prev) {  // (a pair with nothing kept: only the softmax warps act)
             const bool have_cur = e < g.k_top;
             if (have_cur) {
-                if (!wait(smem_u32(&tl->k_empty[ks.idx]), ks.phase ^ 1, tl, 101)) return;
-                load_pair(tk, k_smem + ks.idx * kOperand, smem_u32(&tl->k_full[ks.idx]), it, cur);
+                // a K stage is free once the logits computed from it are complete
+                if (!wait(smem_u32(&tl->s_full[ks.idx]), ks.phase ^ 1, tl, 101)) return;
+                load_k_pair(k_smem + ks.idx * kOperand, smem_u32(&tl->k_full[ks.idx]), it, cur);
                 ks.advance(kKStages);
             }
             if (!q_loaded) {  // behind the pair's first K tiles, which do not depend on the Q buffer
@@ -170,8 +187,9 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
                 q_loaded = true;
             }
             if (have_prev) {
-                if (!wait(smem_u32(&tl->v_empty[vs.idx]), vs.phase ^ 1, tl, 103)) return;
-                load_pair(tv, v_smem + vs.idx * kOperand, smem_u32(&tl->v_full[vs.idx]), it, prev);
+                // a V stage is free once the product computed from it is complete
+                if (!wait(smem_u32(&tl->o_full[vs.idx]), vs.phase ^ 1, tl, 103)) return;
+                load_v_pair(v_smem + vs.idx * kOperand, smem_u32(&tl->v_full[vs.idx]), it, prev);
                 vs.advance(kVStages);
             }
             prev = cur;
@@ -183,16 +201,15 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
     }
 }
 
-// Run by all 32 lanes of its warp, converged: the waits are warp-wide, one elected lane issues.
-__device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned p_smem, unsigned k_smem, unsigned v_smem,
-                         unsigned tmem_base) {
+// The two issuing roles are run by all 32 lanes of their warps, converged: the waits are
+// warp-wide, one elected lane issues.
+
+// S = [Q_0; Q_1] [K_a; K_b]^T for every kept entry.
+__device__ void qk_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_smem, unsigned tmem_base) {
     const Geom &g = P.g;
-    Ring ks, vs, sb, ob, ms;
-    unsigned q_par = 0, p_par = 0;
-    // low descriptor words of the operand buffers; K-major ones ignore the leading offset, the
-    // MN-major V tiles have their two 64-channel halves kHalfTile apart
-    const unsigned q_lo = desc_lo_sw128(q_smem, 16), p_lo = desc_lo_sw128(p_smem, 16), k_lo = desc_lo_sw128(k_smem, 16),
-                   v_lo = desc_lo_sw128(v_smem, kHalfTile);
+    Ring ks, sb, ms;
+    unsigned q_par = 0;
+    const unsigned q_lo = desc_lo_sw128(q_smem, 16), k_lo = desc_lo_sw128(k_smem, 16);
     for (int id = blockIdx.x; id < P.n_items; id += gridDim.x) {
         if (!wait_w(smem_u32(&tl->m_full[ms.idx]), ms.phase, tl, 207)) return;
         const int *rows = tl->rows[ms.idx][0];
@@ -202,60 +219,75 @@ __device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned p_
             if (!wait_w(smem_u32(&tl->q_full), q_par, tl, 201)) return;
             q_par ^= 1;
         }
-        bool have_prev = false;
-        while (e < g.k_top || have_prev) {
-            const bool have_cur = e < g.k_top;
-            if (have_cur) {  // S = [Q_0; Q_1] [K_a; K_b]^T, one chain per K tile
-                if (!wait_w(smem_u32(&tl->k_full[ks.idx]), ks.phase, tl, 202)) return;
-                if (!wait_w(smem_u32(&tl->s_empty[sb.idx]), sb.phase ^ 1, tl, 203)) return;
-                tc_fence_after();
-                const unsigned d_tmem = tmem_base + sb.idx * 128;
-                const unsigned b_lo = k_lo + ks.idx * (kOperand >> 4);
-                e = next_entry(rows, e, g.k_top, &cur);
-                if (elect_one()) {
+        while (e < g.k_top) {
+            e = next_entry(rows, e, g.k_top, &cur);  // (only "is there another entry" matters here)
+            if (!wait_w(smem_u32(&tl->k_full[ks.idx]), ks.phase, tl, 202)) return;
+            if (!wait_w(smem_u32(&tl->s_empty[sb.idx]), sb.phase ^ 1, tl, 203)) return;
+            tc_fence_after();
+            const unsigned d_tmem = tmem_base + sb.idx * 128;
+            const unsigned b_lo = k_lo + ks.idx * (kOperand >> 4);
+            if (elect_one()) {
 #pragma unroll
-                    for (int tile = 0; tile < 2; ++tile)
+                for (int c = 0; c < 2; ++c)
 #pragma unroll
-                        for (int c = 0; c < 2; ++c)
-#pragma unroll
-                            for (int k4 = 0; k4 < 4; ++k4)
-                                tc_mma_bf16_split(d_tmem + tile * 64, q_lo + ((c * 2 * kHalfTile + k4 * 32) >> 4), kHiK,
-                                                  b_lo + ((tile * kTile + c * kHalfTile + k4 * 32) >> 4), kHiK, kIdescQK,
-                                                  (c | k4) != 0);
-                    tc_commit(smem_u32(&tl->s_full[sb.idx]));
-                    tc_commit(smem_u32(&tl->k_empty[ks.idx]));
-                    if (e >= g.k_top) tc_commit(smem_u32(&tl->q_empty));  // that was the pair's last use of Q
-                }
-                __syncwarp();
-                sb.advance(2);
-                ks.advance(kKStages);
+                    for (int k4 = 0; k4 < 4; ++k4)
+                        tc_mma_bf16_split(d_tmem, q_lo + ((c * 2 * kHalfTile + k4 * 32) >> 4), kHiK,
+                                          b_lo + ((c * 2 * kHalfTile + k4 * 32) >> 4), kHiK, kIdescQK, (c | k4) != 0);
+                tc_commit(smem_u32(&tl->s_full[sb.idx]));  // logits ready = K stage free (same ring position)
+                if (e >= g.k_top) tc_commit(smem_u32(&tl->q_empty));  // that was the pair's last use of Q
             }
-            if (have_prev) {  // O = P [V_a; V_b] of the entry before
-                if (!wait_w(smem_u32(&tl->p_full), p_par, tl, 204)) return;
-                p_par ^= 1;
-                if (!wait_w(smem_u32(&tl->v_full[vs.idx]), vs.phase, tl, 205)) return;
-                if (!wait_w(smem_u32(&tl->o_empty[ob.idx]), ob.phase ^ 1, tl, 206)) return;
-                tc_fence_after();
-                const unsigned d_tmem = tmem_base + 256 + ob.idx * 128;
-                const unsigned b_lo = v_lo + vs.idx * (kOperand >> 4);
-                if (elect_one()) {
-#pragma unroll
-                    for (int s = 0; s < 8; ++s)  // 16 keys per step: P column half = V tile = s / 4
-                        tc_mma_bf16_split(d_tmem, p_lo + (((s >> 2) * 2 * kHalfTile + (s & 3) * 32) >> 4), kHiK,
-                                          b_lo + (((s >> 2) * kTile + (s & 3) * 2048) >> 4), kHiK, kIdescPV, s != 0);
-                    tc_commit(smem_u32(&tl->o_full[ob.idx]));
-                    tc_commit(smem_u32(&tl->v_empty[vs.idx]));
-                }
-                __syncwarp();
-                ob.advance(2);
-                vs.advance(kVStages);
-            }
-            have_prev = have_cur;
+            __syncwarp();
+            sb.advance(2);
+            ks.advance(kKStages);
         }
         if (elect_one()) mbar_arrive(smem_u32(&tl->m_empty[ms.idx]));
         __syncwarp();
         ms.advance(kMaskSlots);
     }
+}
+
+// O = P [V_a; V_b] for every kept entry.
+__device__ void pv_role(const Params &P, Tail *tl, unsigned p_smem, unsigned v_smem, unsigned tmem_base) {
+    const Geom &g = P.g;
+    Ring vs, ob, ms;
+    unsigned p_par = 0;
+    // the MN-major V tiles have their two 64-channel halves kHalfTile apart
+    const unsigned p_lo = desc_lo_sw128(p_smem, 16), v_lo = desc_lo_sw128(v_smem, kHalfTile);
+    for (int id = blockIdx.x; id < P.n_items; id += gridDim.x) {
+        if (!wait_w(smem_u32(&tl->m_full[ms.idx]), ms.phase, tl, 208)) return;
+        const int *rows = tl->rows[ms.idx][0];
+        Entry cur;
+        int e = next_entry(rows, -1, g.k_top, &cur);
+        while (e < g.k_top) {
+            e = next_entry(rows, e, g.k_top, &cur);
+            if (!wait_w(smem_u32(&tl->v_full[vs.idx]), vs.phase, tl, 205)) return;
+            if (!wait_w(smem_u32(&tl->p_full), p_par, tl, 204)) return;  // also: O buffer ob has been folded
+            p_par ^= 1;
+            tc_fence_after();
+            const unsigned d_tmem = tmem_base + 256 + ob.idx * 128;
+            const unsigned b_lo = v_lo + vs.idx * (kOperand >> 4);
+            if (elect_one()) {
+#pragma unroll
+                for (int s = 0; s < 8; ++s)  // 16 keys per step: P column half = V tile = s / 4
+                    tc_mma_bf16_split(d_tmem, p_lo + (((s >> 2) * 2 * kHalfTile + (s & 3) * 32) >> 4), kHiK,
+                                      b_lo + (((s >> 2) * kTile + (s & 3) * 2048) >> 4), kHiK, kIdescPV, s != 0);
+                tc_commit(smem_u32(&tl->o_full[ob.idx]));  // product ready = V stage and P buffer free
+            }
+            __syncwarp();
+            ob.advance(2);
+            vs.advance(kVStages);
+        }
+        if (elect_one()) mbar_arrive(smem_u32(&tl->m_empty[ms.idx]));
+        __syncwarp();
+        ms.advance(kMaskSlots);
+    }
+}
+
+// 2^x by the special-function unit (relative error about 2^-22; -inf gives 0).
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
 
 // o[0..63] = o * alpha + O, O being 64 columns of this thread's lane of a TMEM buffer.
@@ -270,8 +302,8 @@ __device__ __forceinline__ void fold_output(float *o, float alpha, unsigned tadd
 
 // Eight softmax warps. Warps w and w + 4 share the 32 TMEM lanes (query tokens) 32 (w % 4) ..: the
 // first takes keys 0..31 of the token's block and output channels 0..63, the second keys 32..63
-// and channels 64..127. The two exchange their partial row maxima (and, at the end, sums)
-// through shared memory, meeting on an mbarrier of their own.
+// and channels 64..127. Both read all 64 logits for the row maximum, so they only have to meet
+// once per pair, to add up their partial sums (through shared memory, on an mbarrier of their own).
 __device__ void softmax_role(const Params &P, Tail *tl, unsigned char *p_ptr, unsigned tmem_base, int t) {
     const Geom &g = P.g;
     const int lane = t & 31, row = t & 127, part = t >> 7, half = row >> 6, mq = row & 63, wq = row >> 5;
@@ -305,14 +337,19 @@ __device__ void softmax_role(const Params &P, Tail *tl, unsigned char *p_ptr, un
         for (int i = 0; i < 64; ++i) o[i] = 0.f;
         float m = -CUDART_INF_F, l = 0.f, alpha_prev = 1.f;
         bool have_prev = false;
-        Entry cur;
+        Entry cur, nxt;
         int e = next_entry(rows, -1, g.k_top, &cur);
         while (e < g.k_top) {
-            // this token's logits against keys 32 part .. 32 part + 31 of its row's key block
+            const int e_next = next_entry(rows, e, g.k_top, &nxt);  // its latency hides behind the wait
+            // this token's 64 logits against its row's key block: both threads of the token read
+            // all of them for the row maximum; each then exponentiates its own 32
             if (!wait(smem_u32(&tl->s_full[sb.idx]), sb.phase, tl, 301)) return;
             tc_fence_after();
-            float sv[32];
-            tmem_ld_32x32(tmem_base + sb.idx * 128 + half * 64 + part * 32 + lane_off, sv);
+            unsigned sr[64];
+            const unsigned s_addr = tmem_base + sb.idx * 128 + half * 64 + lane_off;
+            tmem_ld_32x32_issue(s_addr + part * 32, sr);             // own keys first
+            tmem_ld_32x32_issue(s_addr + (part ^ 1) * 32, sr + 32);  // the partner's
+            tmem_ld_wait();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&tl->s_empty[sb.idx]));
@@ -326,30 +363,30 @@ __device__ void softmax_role(const Params &P, Tail *tl, unsigned char *p_ptr, un
                 if (g.causal) lim = min(lim, tq - k0 + 1);
                 n_hi = (int)max(0ll, min(lim, (long long)kBlk));
             }
-            n_hi -= part * 32;  // in this thread's 32 keys
+            const int n_own = n_hi - part * 32, n_oth = n_hi - (part ^ 1) * 32;  // within each half
             float mx4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
-            if (n_hi >= 32) {
+            if (n_hi == kBlk) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], sv[i]);
+                for (int i = 0; i < 64; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(sr[i]));
             } else {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], i < n_hi ? sv[i] : -CUDART_INF_F);
+                for (int i = 0; i < 32; ++i) {
+                    mx4[i & 3] = fmaxf(mx4[i & 3], i < n_own ? __uint_as_float(sr[i]) : -CUDART_INF_F);
+                    mx4[i & 3] = fmaxf(mx4[i & 3], i < n_oth ? __uint_as_float(sr[32 + i]) : -CUDART_INF_F);
+                }
             }
-            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-            float mx_other;
-            if (!exchange(mx, &mx_other)) return;
-            const float m_new = fmaxf(m, fmaxf(mx, mx_other));
+            const float m_new = fmaxf(m, fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])));
             // with no key allowed so far m_new is -inf: every p is 0 and nothing is rescaled
             const float shift = m_new == -CUDART_INF_F ? 0.f : -m_new * P.scale_log2;
-            const float alpha = m_new == m ? 1.f : exp2f((m - m_new) * P.scale_log2);
+            const float alpha = m_new == m ? 1.f : fast_exp2((m - m_new) * P.scale_log2);
             float sum4[4] = {0.f, 0.f, 0.f, 0.f};
             unsigned packed[16];
 #pragma unroll
             for (int i = 0; i < 32; i += 2) {
-                float p0 = exp2f(fmaf(sv[i], P.scale_log2, shift));
-                float p1 = exp2f(fmaf(sv[i + 1], P.scale_log2, shift));
-                p0 = i < n_hi ? p0 : 0.f;
-                p1 = i + 1 < n_hi ? p1 : 0.f;
+                float p0 = fast_exp2(fmaf(__uint_as_float(sr[i]), P.scale_log2, shift));
+                float p1 = fast_exp2(fmaf(__uint_as_float(sr[i + 1]), P.scale_log2, shift));
+                p0 = i < n_own ? p0 : 0.f;
+                p1 = i + 1 < n_own ? p1 : 0.f;
                 sum4[(i >> 1) & 3] += p0 + p1;
                 __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
                 packed[i >> 1] = *reinterpret_cast<unsigned *>(&pk);
@@ -366,18 +403,17 @@ __device__ void softmax_role(const Params &P, Tail *tl, unsigned char *p_ptr, un
                 *reinterpret_cast<uint4 *>(p_row + (((part * 4 + c) ^ sw) << 4)) =
                     make_uint4(packed[4 * c], packed[4 * c + 1], packed[4 * c + 2], packed[4 * c + 3]);
             fence_async_smem();
+            tc_fence_before();  // this thread's TMEM reads (the product folded last round) are done
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&tl->p_full));
             if (have_prev) {
                 fold_output(o, alpha_prev, tmem_base + 256 + ob.idx * 128 + part * 64 + lane_off);
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&tl->o_empty[ob.idx]));
                 ob.advance(2);
             }
             alpha_prev = alpha;
             have_prev = true;
-            e = next_entry(rows, e, g.k_top, &cur);
+            e = e_next;
+            cur = nxt;
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&tl->m_empty[ms.idx]));
@@ -386,9 +422,6 @@ __device__ void softmax_role(const Params &P, Tail *tl, unsigned char *p_ptr, un
             if (!wait(smem_u32(&tl->o_full[ob.idx]), ob.phase, tl, 303)) return;
             tc_fence_after();
             fold_output(o, alpha_prev, tmem_base + 256 + ob.idx * 128 + part * 64 + lane_off);
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&tl->o_empty[ob.idx]));
             ob.advance(2);
         }
         float l_other;
@@ -424,15 +457,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     if (threadIdx.x == 0) {
         mbar_init(smem_u32(&tl->q_full), 1);
         mbar_init(smem_u32(&tl->q_empty), 1);
-        for (int i = 0; i < kKStages; ++i) { mbar_init(smem_u32(&tl->k_full[i]), 1); mbar_init(smem_u32(&tl->k_empty[i]), 1); }
-        for (int i = 0; i < kVStages; ++i) { mbar_init(smem_u32(&tl->v_full[i]), 1); mbar_init(smem_u32(&tl->v_empty[i]), 1); }
+        for (int i = 0; i < kKStages; ++i) mbar_init(smem_u32(&tl->k_full[i]), 1);
+        for (int i = 0; i < kVStages; ++i) mbar_init(smem_u32(&tl->v_full[i]), 1);
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&tl->s_full[i]), 1); mbar_init(smem_u32(&tl->s_empty[i]), 8);
-            mbar_init(smem_u32(&tl->o_full[i]), 1); mbar_init(smem_u32(&tl->o_empty[i]), 8);
+            mbar_init(smem_u32(&tl->o_full[i]), 1);
         }
         mbar_init(smem_u32(&tl->p_full), 8);
         for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&tl->x_bar[i]), 2);
-        for (int i = 0; i < kMaskSlots; ++i) { mbar_init(smem_u32(&tl->m_full[i]), 1); mbar_init(smem_u32(&tl->m_empty[i]), 10); }
+        for (int i = 0; i < kMaskSlots; ++i) { mbar_init(smem_u32(&tl->m_full[i]), 1); mbar_init(smem_u32(&tl->m_empty[i]), 11); }
         tl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -449,10 +482,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     if (warp == 0) {
         if (lane == 0) producer_role(P, &tmap_q, &tmap_k, &tmap_v, tl, q_smem, k_smem, v_smem);
     } else if (warp == 1) {
-        mma_role(P, tl, q_smem, p_smem, k_smem, v_smem, tmem_base);
+        qk_role(P, tl, q_smem, k_smem, tmem_base);
     } else if (warp == 2) {
         mask_loader_role(P, tl, lane);
-    } else if (warp >= 4) {
+    } else if (warp == 3) {
+        pv_role(P, tl, p_smem, v_smem, tmem_base);
+    } else {
         softmax_role(P, tl, smem + kOperand, tmem_base, (int)threadIdx.x - 128);
     }
     __syncwarp();
@@ -486,7 +521,7 @@ stream_status launch_attn_tc(const Geom &g, const void *q, const void *k, const 
     CUtensorMap tq, tk, tv;
     stream_status rc = make_map5_bf16_d128(&tq, q, g.T, g.H, g.batch, g.qs_t, g.qs_h, g.qs_b, 2, "q");
     if (rc != STREAM_OK) return rc;
-    rc = make_map5_bf16_d128(&tk, k, g.T, g.G, g.batch, g.ks_t, g.ks_h, g.ks_b, 1, "k");
+    rc = make_map_bf16_d128(&tk, k, g.T, g.G, g.batch, g.ks_t, g.ks_h, g.ks_b, "k");  // 4-D: 64 x 64 half tiles
     if (rc != STREAM_OK) return rc;
     rc = make_map5_bf16_d128(&tv, v, g.T, g.G, g.batch, g.ks_t, g.ks_h, g.ks_b, 1, "v");
     if (rc != STREAM_OK) return rc;

@@ -36,7 +36,8 @@ typedef enum {
     STREAM_ERR_UNSUPPORTED = 2, /* valid request that no kernel here covers (see stream_problem) */
     STREAM_ERR_WORKSPACE = 3,   /* workspace or staging buffer missing, misaligned or too small */
     STREAM_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed; text in stream_last_error */
-    STREAM_ERR_DEVICE_CHECK = 5 /* a kernel gave up on a bounded wait; see stream_read_stats */
+    STREAM_ERR_DEVICE_CHECK = 5 /* a kernel gave up on a bounded wait or met an out-of-range mask
+                                   entry; see stream_read_stats */
 } stream_status;
 
 typedef enum { STREAM_F32 = 0, STREAM_BF16 = 1 } stream_dtype;
@@ -148,9 +149,35 @@ stream_status stream_sparse_attention(const stream_problem *p, const void *q, co
                                       const int32_t *mask, float scale, void *out, void *cuda_stream);
 
 /*
+ * Vertical attention scores of a mask and their kurtosis (Section 4.1 of the paper: the column
+ * sums of a head's sparse mask show which key blocks attract the later queries; heads whose
+ * vertical scores have a high kurtosis are the "receiver heads").
+ *
+ *   vertical[b, h, r] = sum over the head's query blocks q and slots j with mask[b, h, q, j] == r
+ *                       of scores[b, h, q, j]   (of 1 if scores is NULL: the binary mask)
+ *   kurtosis[b, h]    = m4 / m2^2 of vertical[b, h, :], m2 and m4 the second and fourth central
+ *                       moments over the ceil(T / block_k) key blocks (Pearson, not excess); 0
+ *                       if all vertical scores of the head are equal
+ *
+ *   mask          device int32 [batch, n_q_heads, ceil(T/block_q), k_top]; entries < 0 are skipped
+ *   scores        device float32, same shape (score_out of stream_build_mask), or NULL; -inf
+ *                 padding is never read because its mask entry is < 0
+ *   vertical_out  device float32 [batch, n_q_heads, ceil(T/block_k)]; overwritten
+ *   kurtosis_out  device float32 [batch, n_q_heads], or NULL
+ *   workspace     as for stream_build_mask; stream_read_stats afterwards returns
+ *                 STREAM_ERR_DEVICE_CHECK if a mask entry was >= ceil(T/block_k) (such entries
+ *                 are ignored). Sums are fp32 and added in no fixed order.
+ * Only T, block_k, block_q, k_top, batch and n_q_heads of *p matter. Up to 49152 key blocks per
+ * head; more gives STREAM_ERR_UNSUPPORTED.
+ */
+stream_status stream_vertical_scores(const stream_problem *p, const int32_t *mask, const float *scores, float *vertical_out,
+                                     float *kurtosis_out, void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
  * Synchronous read-back of the counters left by the last stream_build_mask that used this
  * workspace. Waits for `cuda_stream` to drain, copies the header to *out (HOST pointer) and
- * returns STREAM_ERR_DEVICE_CHECK if the kernel recorded a bounded wait that ran out.
+ * returns STREAM_ERR_DEVICE_CHECK if the kernel recorded a failed device-side check (a bounded
+ * wait that ran out; an out-of-range mask entry in stream_vertical_scores).
  */
 stream_status stream_read_stats(const void *workspace, stream_stats *out, void *cuda_stream);
 

@@ -8,4 +8,5 @@ from .stream_oracle import (  # noqa: F401
     sparse_attention_rows,
     threads,
     tile_score,
+    vertical_scores,
 )

@@ -319,3 +319,49 @@ int so_sparse_attention_rows(const so_problem *p, const void *Q, const void *K, 
     }
     return err;
 }
+
+/*
+ * Vertical attention scores of a block mask and their kurtosis (Section 4.1: receiver heads are
+ * the heads whose vertical scores have high kurtosis, i.e. a few key blocks take most of the
+ * attention of the later queries).
+ *   mask   [batch * n_q_heads * n_query_blocks, k]  as produced by so_build_mask_rows for all rows
+ *   score  same shape or NULL: weight of each kept block (NULL: every kept block counts 1)
+ *   vertical_out [batch * n_q_heads, n_key_blocks]  v[h, r] = sum over query blocks q and slots j
+ *                                                   with mask[h, q, j] == r of the weight
+ *   kurtosis_out [batch * n_q_heads]  m4 / m2^2 of v[h, :] (central moments over the n_key_blocks
+ *                                     columns, not excess); 0 when the scores are all equal
+ * Everything in fp64, in index order. n_key_blocks = ceil(T / b_k).
+ */
+int so_vertical_scores(const so_problem *p, const int32_t *mask, const float *score, double *vertical_out,
+                       double *kurtosis_out) {
+    int rc = check_problem(p);
+    if (rc) return rc;
+    const int64_t Nq = so_num_query_blocks(p), Nk = (p->T + p->block_k - 1) / p->block_k;
+    const int64_t heads = (int64_t)p->batch * p->n_q_heads;
+    for (int64_t h = 0; h < heads; ++h) {
+        double *v = vertical_out + h * Nk;
+        for (int64_t r = 0; r < Nk; ++r) v[r] = 0.0;
+        for (int64_t q = 0; q < Nq; ++q)
+            for (int64_t j = 0; j < p->k_top; ++j) {
+                int64_t at = (h * Nq + q) * p->k_top + j;
+                int32_t r = mask[at];
+                if (r < 0) continue;
+                if (r >= Nk) return -4;
+                v[r] += score ? (double)score[at] : 1.0;
+            }
+        if (kurtosis_out) {
+            double mean = 0.0, m2 = 0.0, m4 = 0.0;
+            for (int64_t r = 0; r < Nk; ++r) mean += v[r];
+            mean /= (double)Nk;
+            for (int64_t r = 0; r < Nk; ++r) {
+                double dlt = v[r] - mean;
+                m2 += dlt * dlt;
+                m4 += dlt * dlt * dlt * dlt;
+            }
+            m2 /= (double)Nk;
+            m4 /= (double)Nk;
+            kurtosis_out[h] = m2 > 0.0 ? m4 / (m2 * m2) : 0.0;
+        }
+    }
+    return 0;
+}

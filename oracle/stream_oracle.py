@@ -104,6 +104,8 @@ def _load():
         lib.so_sparse_attention_rows.restype = ctypes.c_int
         lib.so_sparse_attention_rows.argtypes = [ctypes.POINTER(_CProblem), vp, vp, vp, i64p, ctypes.c_int64,
                                                  vp, ctypes.c_double, vp]
+        lib.so_vertical_scores.restype = ctypes.c_int
+        lib.so_vertical_scores.argtypes = [ctypes.POINTER(_CProblem), vp, vp, vp, vp]
         _lib = lib
     return _lib
 
@@ -178,3 +180,27 @@ def sparse_attention_rows(p: OracleProblem, q: np.ndarray, k: np.ndarray, v: np.
     if rc:
         raise RuntimeError(f"so_sparse_attention_rows failed with {rc}")
     return out
+
+
+def vertical_scores(p: OracleProblem, mask: np.ndarray, scores: np.ndarray | None = None):
+    """Column sums of a block mask (binary, or weighted by ``scores``) per head and their kurtosis.
+
+    ``mask`` (and ``scores``) cover every row: [num_rows, k_top]. Returns (vertical fp64
+    [batch * n_q_heads, ceil(T / block_k)], kurtosis fp64 [batch * n_q_heads]).
+    """
+    lib = _load()
+    n = num_rows(p)
+    mask = np.ascontiguousarray(mask, dtype=np.int32)
+    if mask.shape != (n, p.k_top):
+        raise ValueError(f"mask: need shape {(n, p.k_top)}, got {mask.shape}")
+    if scores is not None:
+        scores = np.ascontiguousarray(scores, dtype=np.float32)
+        if scores.shape != mask.shape:
+            raise ValueError("scores must have the mask's shape")
+    heads, nk = p.batch * p.n_q_heads, -(-p.T // p.block_k)
+    vert = np.empty((heads, nk), np.float64)
+    kurt = np.empty((heads,), np.float64)
+    rc = lib.so_vertical_scores(ctypes.byref(p.c()), _ptr(mask), _ptr(scores), _ptr(vert), _ptr(kurt))
+    if rc:
+        raise RuntimeError(f"so_vertical_scores failed with {rc}")
+    return vert, kurt

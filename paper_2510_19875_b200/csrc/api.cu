@@ -159,10 +159,27 @@ stream_status stream_read_stats(const void *workspace, stream_stats *out, void *
     e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
     if (out->error != 0) {
-        set_error("kernel gave up on a bounded wait: code %u, info %u", out->error, out->error_info);
+        set_error("a kernel recorded a failed device-side check: code %u, info %u", out->error, out->error_info);
         return STREAM_ERR_DEVICE_CHECK;
     }
     return STREAM_OK;
+}
+
+stream_status stream_vertical_scores(const stream_problem *p, const int32_t *mask, const float *scores, float *vertical_out,
+                                     float *kurtosis_out, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    Geom g;
+    stream_status rc = make_geom(p, &g);
+    if (rc != STREAM_OK) return rc;
+    if (mask == nullptr || vertical_out == nullptr) { set_error("mask and vertical_out must not be NULL"); return STREAM_ERR_INVALID_ARG; }
+    if (workspace == nullptr || workspace_bytes < sizeof(WorkspaceHeader) || ((uintptr_t)workspace & 255) != 0) {
+        set_error("workspace must be a 256-byte aligned device buffer of at least %zu bytes", sizeof(WorkspaceHeader));
+        return STREAM_ERR_WORKSPACE;
+    }
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    WorkspaceHeader *ws = (WorkspaceHeader *)workspace;
+    cudaError_t e = cudaMemsetAsync(ws, 0, sizeof(WorkspaceHeader), st);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(workspace)");
+    return launch_vertical(g, mask, scores, vertical_out, kurtosis_out, &ws->error, st);
 }
 
 stream_status stream_check_device_status(void *cuda_stream) {

@@ -44,27 +44,28 @@ constexpr int kBlk = 64, kD = 128;
 constexpr int kHalfTile = kBlk * 128;       // 64 rows x 128 bytes
 constexpr int kTile = 2 * kHalfTile;        // one 64 x 128 tile
 constexpr int kOperand = 2 * kTile;         // two tiles (K_a, K_b or V_a, V_b), or a 128-row operand
-constexpr int kKStages = 2, kVStages = 2;   // = S and O buffers (see Tail)
+constexpr int kMaxKStages = 3, kVStages = 2;  // K stages: 3 if shared memory allows, else 2; V stages = O buffers
 constexpr int kMaskSlots = 2;               // pairs whose mask rows are resident
 constexpr int kMaxKTopTc = 1024;
 
 struct Tail {
     unsigned long long q_full, q_empty;
-    unsigned long long k_full[kKStages], v_full[kVStages];
-    // s_full also tells the producer that K stage i is free, o_full that V stage i is: the rings
-    // of K stages and S buffers (V stages and O buffers) have the same length and move together.
-    // There is no "o_empty": P of entry j is published (p_full) after the same threads folded the
-    // product of entry j - 2, and the P V warp waits for every P before it overwrites that buffer.
+    unsigned long long k_full[kMaxKStages], k_empty[kMaxKStages], v_full[kVStages];
+    // o_full also tells the producer that V stage i is free: the rings of V stages and O buffers
+    // have the same length and move together. There is no "o_empty": P of entry j is published
+    // (p_full) after the same threads folded the product of entry j - 2, and the P V warp waits
+    // for every P before it overwrites that buffer.
     unsigned long long s_full[2], s_empty[2], o_full[2], p_full;
     unsigned long long m_full[kMaskSlots], m_empty[kMaskSlots];
     unsigned long long x_bar[4];  // softmax warps w and w + 4 meet here
     unsigned int tmem_base;
     int abort_flag;
     float xch[2][128][2];         // their exchange slots: [buffer][token][part]
-    int rows[kMaskSlots][2][kMaxKTopTc];  // mask rows of the resident pairs (-1 where a row has nothing)
 };
-constexpr int kSmemBytes = (2 + kKStages + kVStages) * kOperand + (int)sizeof(Tail) + 1024;
-static_assert(kSmemBytes <= 232448, "exceeds the shared memory of one CTA");
+// Dynamic shared memory: Q | P | V stages | K stages | Tail | mask rows [kMaskSlots][2][row_stride]
+// (-1 where a row has nothing), the first four 1024-byte aligned.
+constexpr int kFixedOperands = 2 + kVStages;
+constexpr int kMaxSmemPerCta = 232448;
 
 constexpr unsigned kIdescQK = idesc_bf16(128, 128, false);  // B = stacked K tiles, K-major
 constexpr unsigned kIdescPV = idesc_bf16(128, 128, true);   // B = stacked V tiles, MN-major
@@ -73,6 +74,9 @@ constexpr unsigned kHiK = desc_hi_sw128(1024);              // every operand: 8-
 struct Params {
     Geom g;
     int n_items, n_pairs;  // pairs per kv head: ceil(hpg / 2)
+    int row_stride;        // ints per resident mask row (k_top rounded up to a multiple of 4)
+    int smem_bytes;        // dynamic shared memory of the launch
+    int n_k_stages;        // set by the kernel from what fits behind its aligned base
     const int32_t *mask;
     __nv_bfloat16 *out;
     float scale_log2;      // logit scale times log2(e)
@@ -85,6 +89,11 @@ __device__ __forceinline__ bool wait(unsigned bar, unsigned parity, Tail *tl, un
 // The same for a whole converged warp (all lanes get the same answer).
 __device__ __forceinline__ bool wait_w(unsigned bar, unsigned parity, Tail *tl, unsigned code) {
     return mbar_wait_warp(bar, parity, &tl->abort_flag, &g_attn_status[0], &g_attn_status[1], code);
+}
+
+// Shared copy of the mask rows of the pair in slot `slot`: [2][row_stride] ints behind the Tail.
+__device__ __forceinline__ int *mask_rows(Tail *tl, const Params &P, int slot) {
+    return reinterpret_cast<int *>(tl + 1) + slot * 2 * P.row_stride;
 }
 
 // The pair a CTA works on in its n-th round.
@@ -108,12 +117,12 @@ __device__ __forceinline__ Item decode_item(const Params &P, int id) {
 }
 
 // Entry e of the two rows: key block per row (negative = this row has nothing at e). An entry
-// is processed if either row has a block there. `rows` is the pair's shared copy [2][kMaxKTopTc].
+// is processed if either row has a block there. `rows` is the pair's shared copy [2][stride].
 struct Entry { int a, b; };
-__device__ __forceinline__ int next_entry(const int *rows, int e, int k_top, Entry *x) {
+__device__ __forceinline__ int next_entry(const int *rows, int stride, int e, int k_top, Entry *x) {
     for (++e; e < k_top; ++e) {
         x->a = rows[e];
-        x->b = rows[kMaxKTopTc + e];
+        x->b = rows[stride + e];
         if (x->a >= 0 || x->b >= 0) return e;
     }
     return k_top;
@@ -131,10 +140,10 @@ __device__ void mask_loader_role(const Params &P, Tail *tl, int lane) {
         if (!wait(smem_u32(&tl->m_empty[ms.idx]), ms.phase ^ 1, tl, 401)) return;
         const int32_t *m0 = P.mask + (((long long)it.b * g.H + it.h0) * g.n_qb + it.qb) * g.k_top;
         const int32_t *m1 = m0 + (long long)g.n_qb * g.k_top;
-        int *dst = tl->rows[ms.idx][0];
+        int *dst = mask_rows(tl, P, ms.idx);
         for (int e = lane; e < g.k_top; e += 32) {
             dst[e] = __ldg(m0 + e);
-            dst[kMaxKTopTc + e] = it.R == 2 ? __ldg(m1 + e) : -1;
+            dst[P.row_stride + e] = it.R == 2 ? __ldg(m1 + e) : -1;
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&tl->m_full[ms.idx]));
@@ -142,11 +151,26 @@ __device__ void mask_loader_role(const Params &P, Tail *tl, int lane) {
     }
 }
 
+// One thread feeds two independent streams of TMA loads, the K tiles (with each pair's Q tiles)
+// and the V tiles, each as far ahead as its ring of stages allows. It never blocks on one stream
+// while the other could move: every step probes its barrier without waiting.
+struct LoadStream {
+    int id;            // pair being walked
+    int e;             // current entry (k_top = pair exhausted), -2 = pair not opened yet
+    int n_issued;      // loads issued for this pair
+    Entry cur;
+    Ring ring, ms;
+    bool q_due;        // (K stream) the pair's Q tiles still have to be requested
+};
+
 __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUtensorMap *tk, const CUtensorMap *tv,
                               Tail *tl, unsigned q_smem, unsigned k_smem, unsigned v_smem) {
     const Geom &g = P.g;
-    Ring ks, vs, ms;
     unsigned q_par = 0;
+    LoadStream K, V;
+    K.id = V.id = blockIdx.x;
+    K.e = V.e = -2;
+    K.q_due = V.q_due = false;
     // a row without a block at an entry gets block 0; its logits are masked out entirely
     auto load_k_pair = [&](unsigned dst, unsigned bar, const Item &it, Entry x) {  // [half][tile][64 rows][128 B]
         const int ba = x.a >= 0 ? x.a : 0, bb = x.b >= 0 ? x.b : 0;
@@ -163,41 +187,64 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
         tma_load_5d(dst, tv, bar, 0, ba * kBlk, it.kvh, 0, it.b);
         tma_load_5d(dst + kTile, tv, bar, 0, bb * kBlk, it.kvh, 0, it.b);
     };
-    for (int id = blockIdx.x; id < P.n_items; id += gridDim.x) {
-        const Item it = decode_item(P, id);
-        if (!wait(smem_u32(&tl->m_full[ms.idx]), ms.phase, tl, 104)) return;
-        const int *rows = tl->rows[ms.idx][0];
-        Entry cur, prev;
-        int e = next_entry(rows, -1, g.k_top, &cur);
-        bool q_loaded = false, have_prev = false;
-        while (e < g.k_top || have_prev) {  // (a pair with nothing kept: only the softmax warps act)
-            const bool have_cur = e < g.k_top;
-            if (have_cur) {
-                // a K stage is free once the logits computed from it are complete
-                if (!wait(smem_u32(&tl->s_full[ks.idx]), ks.phase ^ 1, tl, 101)) return;
-                load_k_pair(k_smem + ks.idx * kOperand, smem_u32(&tl->k_full[ks.idx]), it, cur);
-                ks.advance(kKStages);
-            }
-            if (!q_loaded) {  // behind the pair's first K tiles, which do not depend on the Q buffer
-                if (!wait(smem_u32(&tl->q_empty), q_par ^ 1, tl, 102)) return;
-                q_par ^= 1;
-                const unsigned bar = smem_u32(&tl->q_full);
-                mbar_arrive_expect_tx(bar, (unsigned)kOperand);
-                tma_load_5d(q_smem, tq, bar, 0, it.qb * kBlk, it.h0, 0, it.b);  // heads h0 and h0 + 1
-                q_loaded = true;
-            }
-            if (have_prev) {
-                // a V stage is free once the product computed from it is complete
-                if (!wait(smem_u32(&tl->o_full[vs.idx]), vs.phase ^ 1, tl, 103)) return;
-                load_v_pair(v_smem + vs.idx * kOperand, smem_u32(&tl->v_full[vs.idx]), it, prev);
-                vs.advance(kVStages);
-            }
-            prev = cur;
-            have_prev = have_cur;
-            if (have_cur) e = next_entry(rows, e, g.k_top, &cur);
+    // One step of a stream; true if it did something. is_k selects the K (+ Q) or the V stream.
+    auto step = [&](LoadStream &S, bool is_k) -> bool {
+        if (S.id >= P.n_items) return false;
+        const int *rows = mask_rows(tl, P, S.ms.idx);
+        if (S.e == -2) {  // open the pair: its mask rows must be resident
+            if (!mbar_test_wait(smem_u32(&tl->m_full[S.ms.idx]), S.ms.phase)) return false;
+            S.e = next_entry(rows, P.row_stride, -1, g.k_top, &S.cur);
+            S.q_due = is_k && S.e < g.k_top;  // (a pair with nothing kept: only the softmax warps act)
+            S.n_issued = 0;
+            return true;
         }
-        mbar_arrive(smem_u32(&tl->m_empty[ms.idx]));
-        ms.advance(kMaskSlots);
+        if (S.e >= g.k_top && !S.q_due) {  // pair exhausted: give its mask rows back, go to the next one
+            mbar_arrive(smem_u32(&tl->m_empty[S.ms.idx]));
+            S.ms.advance(kMaskSlots);
+            S.id += gridDim.x;
+            S.e = -2;
+            return true;
+        }
+        const Item it = decode_item(P, S.id);
+        if (is_k) {
+            if (S.e < g.k_top && !(S.q_due && S.n_issued > 0)) {
+                // a K stage is free once the logits computed from it are complete
+                if (!mbar_test_wait(smem_u32(&tl->k_empty[S.ring.idx]), S.ring.phase ^ 1)) return false;
+                load_k_pair(k_smem + S.ring.idx * kOperand, smem_u32(&tl->k_full[S.ring.idx]), it, S.cur);
+                S.ring.advance(P.n_k_stages);
+                S.e = next_entry(rows, P.row_stride, S.e, g.k_top, &S.cur);
+                ++S.n_issued;
+                return true;
+            }
+            // Q goes behind the pair's first K tiles, which do not depend on the Q buffer
+            if (!mbar_test_wait(smem_u32(&tl->q_empty), q_par ^ 1)) return false;
+            q_par ^= 1;
+            const unsigned bar = smem_u32(&tl->q_full);
+            mbar_arrive_expect_tx(bar, (unsigned)kOperand);
+            tma_load_5d(q_smem, tq, bar, 0, it.qb * kBlk, it.h0, 0, it.b);  // heads h0 and h0 + 1
+            S.q_due = false;
+            return true;
+        }
+        // a V stage is free once the product computed from it is complete
+        if (!mbar_test_wait(smem_u32(&tl->o_full[S.ring.idx]), S.ring.phase ^ 1)) return false;
+        load_v_pair(v_smem + S.ring.idx * kOperand, smem_u32(&tl->v_full[S.ring.idx]), it, S.cur);
+        S.ring.advance(kVStages);
+        S.e = next_entry(rows, P.row_stride, S.e, g.k_top, &S.cur);
+        return true;
+    };
+    long long t_last = clock64();
+    while (K.id < P.n_items || V.id < P.n_items) {
+        const bool moved_k = step(K, true), moved_v = step(V, false);
+        if (moved_k || moved_v) {
+            t_last = clock64();
+        } else {
+            if (*(volatile int *)&tl->abort_flag) return;
+            if (clock64() - t_last > kWaitCycles) {
+                *(volatile int *)&tl->abort_flag = 1;
+                if (atomicCAS(&g_attn_status[0], 0u, 101u) == 0u) g_attn_status[1] = blockIdx.x;
+                return;
+            }
+        }
     }
 }
 
@@ -212,15 +259,15 @@ __device__ void qk_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_s
     const unsigned q_lo = desc_lo_sw128(q_smem, 16), k_lo = desc_lo_sw128(k_smem, 16);
     for (int id = blockIdx.x; id < P.n_items; id += gridDim.x) {
         if (!wait_w(smem_u32(&tl->m_full[ms.idx]), ms.phase, tl, 207)) return;
-        const int *rows = tl->rows[ms.idx][0];
+        const int *rows = mask_rows(tl, P, ms.idx);
         Entry cur;
-        int e = next_entry(rows, -1, g.k_top, &cur);
+        int e = next_entry(rows, P.row_stride, -1, g.k_top, &cur);
         if (e < g.k_top) {
             if (!wait_w(smem_u32(&tl->q_full), q_par, tl, 201)) return;
             q_par ^= 1;
         }
         while (e < g.k_top) {
-            e = next_entry(rows, e, g.k_top, &cur);  // (only "is there another entry" matters here)
+            e = next_entry(rows, P.row_stride, e, g.k_top, &cur);  // (only "is there another entry" matters here)
             if (!wait_w(smem_u32(&tl->k_full[ks.idx]), ks.phase, tl, 202)) return;
             if (!wait_w(smem_u32(&tl->s_empty[sb.idx]), sb.phase ^ 1, tl, 203)) return;
             tc_fence_after();
@@ -233,12 +280,13 @@ __device__ void qk_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_s
                     for (int k4 = 0; k4 < 4; ++k4)
                         tc_mma_bf16_split(d_tmem, q_lo + ((c * 2 * kHalfTile + k4 * 32) >> 4), kHiK,
                                           b_lo + ((c * 2 * kHalfTile + k4 * 32) >> 4), kHiK, kIdescQK, (c | k4) != 0);
-                tc_commit(smem_u32(&tl->s_full[sb.idx]));  // logits ready = K stage free (same ring position)
+                tc_commit(smem_u32(&tl->s_full[sb.idx]));
+                tc_commit(smem_u32(&tl->k_empty[ks.idx]));
                 if (e >= g.k_top) tc_commit(smem_u32(&tl->q_empty));  // that was the pair's last use of Q
             }
             __syncwarp();
             sb.advance(2);
-            ks.advance(kKStages);
+            ks.advance(P.n_k_stages);
         }
         if (elect_one()) mbar_arrive(smem_u32(&tl->m_empty[ms.idx]));
         __syncwarp();
@@ -255,11 +303,11 @@ __device__ void pv_role(const Params &P, Tail *tl, unsigned p_smem, unsigned v_s
     const unsigned p_lo = desc_lo_sw128(p_smem, 16), v_lo = desc_lo_sw128(v_smem, kHalfTile);
     for (int id = blockIdx.x; id < P.n_items; id += gridDim.x) {
         if (!wait_w(smem_u32(&tl->m_full[ms.idx]), ms.phase, tl, 208)) return;
-        const int *rows = tl->rows[ms.idx][0];
+        const int *rows = mask_rows(tl, P, ms.idx);
         Entry cur;
-        int e = next_entry(rows, -1, g.k_top, &cur);
+        int e = next_entry(rows, P.row_stride, -1, g.k_top, &cur);
         while (e < g.k_top) {
-            e = next_entry(rows, e, g.k_top, &cur);
+            e = next_entry(rows, P.row_stride, e, g.k_top, &cur);
             if (!wait_w(smem_u32(&tl->v_full[vs.idx]), vs.phase, tl, 205)) return;
             if (!wait_w(smem_u32(&tl->p_full), p_par, tl, 204)) return;  // also: O buffer ob has been folded
             p_par ^= 1;
@@ -331,16 +379,16 @@ __device__ void softmax_role(const Params &P, Tail *tl, unsigned char *p_ptr, un
         const long long tq = (long long)it.qb * kBlk + mq;
         const bool row_active = half < it.R && tq < g.T;
         if (!wait(smem_u32(&tl->m_full[ms.idx]), ms.phase, tl, 305)) return;
-        const int *rows = tl->rows[ms.idx][0];
+        const int *rows = mask_rows(tl, P, ms.idx);
         float o[64];
 #pragma unroll
         for (int i = 0; i < 64; ++i) o[i] = 0.f;
         float m = -CUDART_INF_F, l = 0.f, alpha_prev = 1.f;
         bool have_prev = false;
         Entry cur, nxt;
-        int e = next_entry(rows, -1, g.k_top, &cur);
+        int e = next_entry(rows, P.row_stride, -1, g.k_top, &cur);
         while (e < g.k_top) {
-            const int e_next = next_entry(rows, e, g.k_top, &nxt);  // its latency hides behind the wait
+            const int e_next = next_entry(rows, P.row_stride, e, g.k_top, &nxt);  // its latency hides behind the wait
             // this token's 64 logits against its row's key block: both threads of the token read
             // all of them for the row maximum; each then exponentiates its own 32
             if (!wait(smem_u32(&tl->s_full[sb.idx]), sb.phase, tl, 301)) return;
@@ -446,18 +494,21 @@ __device__ void softmax_role(const Params &P, Tail *tl, unsigned char *p_ptr, un
 
 __global__ void __launch_bounds__(kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
-               const __grid_constant__ CUtensorMap tmap_v, Params P) {
+               const __grid_constant__ CUtensorMap tmap_v, Params P) {  // P by value: n_k_stages is filled in here
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char *smem = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    const unsigned q_smem = smem_u32(smem), p_smem = q_smem + kOperand, k_smem = p_smem + kOperand,
-                   v_smem = k_smem + kKStages * kOperand;
-    Tail *tl = (Tail *)(smem + (2 + kKStages + kVStages) * kOperand);
+    // what is left behind the aligned base decides the number of K stages (the same in every thread)
+    const int fixed_bytes = (int)(smem - smem_raw) + (int)sizeof(Tail) + kMaskSlots * 2 * P.row_stride * (int)sizeof(int);
+    P.n_k_stages = min(kMaxKStages, (P.smem_bytes - fixed_bytes) / kOperand - kFixedOperands);
+    const unsigned q_smem = smem_u32(smem), p_smem = q_smem + kOperand, v_smem = p_smem + kOperand,
+                   k_smem = v_smem + kVStages * kOperand;
+    Tail *tl = (Tail *)(smem + (kFixedOperands + P.n_k_stages) * kOperand);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
         mbar_init(smem_u32(&tl->q_full), 1);
         mbar_init(smem_u32(&tl->q_empty), 1);
-        for (int i = 0; i < kKStages; ++i) mbar_init(smem_u32(&tl->k_full[i]), 1);
+        for (int i = 0; i < kMaxKStages; ++i) { mbar_init(smem_u32(&tl->k_full[i]), 1); mbar_init(smem_u32(&tl->k_empty[i]), 1); }
         for (int i = 0; i < kVStages; ++i) mbar_init(smem_u32(&tl->v_full[i]), 1);
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&tl->s_full[i]), 1); mbar_init(smem_u32(&tl->s_empty[i]), 8);
@@ -465,7 +516,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         }
         mbar_init(smem_u32(&tl->p_full), 8);
         for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&tl->x_bar[i]), 2);
-        for (int i = 0; i < kMaskSlots; ++i) { mbar_init(smem_u32(&tl->m_full[i]), 1); mbar_init(smem_u32(&tl->m_empty[i]), 11); }
+        for (int i = 0; i < kMaskSlots; ++i) { mbar_init(smem_u32(&tl->m_full[i]), 1); mbar_init(smem_u32(&tl->m_empty[i]), 12); }
         tl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -535,10 +586,22 @@ stream_status launch_attn_tc(const Geom &g, const void *q, const void *k, const 
     P.scale_log2 = scale * 1.4426950408889634f;
     const int n_sm = sm_count();
     if (n_sm <= 0) { set_error("cannot read the SM count of the current device"); return STREAM_ERR_CUDA; }
-    cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    // room for three K stages if the mask rows are short enough, else two; 1 KB of slack for the
+    // alignment of the base (the kernel counts its stages from what it really gets)
+    P.row_stride = (g.k_top + 3) & ~3;
+    const int tail_bytes = (int)sizeof(Tail) + kMaskSlots * 2 * P.row_stride * (int)sizeof(int);
+    int smem_bytes = (kFixedOperands + kMaxKStages) * kOperand + tail_bytes + 1024;
+    if (smem_bytes > kMaxSmemPerCta) smem_bytes = kMaxSmemPerCta;
+    if (smem_bytes < (kFixedOperands + 2) * kOperand + tail_bytes + 1024) {
+        set_error("tensor-core attention kernel: k_top = %d needs more shared memory than one CTA has", g.k_top);
+        return STREAM_ERR_UNSUPPORTED;
+    }
+    P.smem_bytes = smem_bytes;
+    P.n_k_stages = 0;
+    cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmemPerCta);
     if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(attn_tc)");
     const int grid = (int)(n_items < n_sm ? n_items : n_sm);
-    attn_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(tq, tk, tv, P);
+    attn_tc_kernel<<<grid, kThreads, smem_bytes, st>>>(tq, tk, tv, P);
     e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "attn_tc launch");
     return STREAM_OK;

@@ -47,6 +47,9 @@ stream_status launch_mask_tc(const Geom &g, const void *q, const void *k, int32_
 bool attn_tc_supported(const Geom &g, int dtype);
 stream_status launch_attn_tc(const Geom &g, const void *q, const void *k, const void *v, const int32_t *mask,
                              float scale, void *out, cudaStream_t st);
+// bad_flag: device word that gets bit 0 set if a mask entry is >= the number of key blocks.
+stream_status launch_vertical(const Geom &g, const int32_t *mask, const float *score, float *vertical, float *kurtosis,
+                              unsigned int *bad_flag, cudaStream_t st);
 // Drains `st` and copies the tensor-core attention kernel's status words (code, block) to out.
 stream_status read_attn_status(unsigned int out[2], cudaStream_t st);
 

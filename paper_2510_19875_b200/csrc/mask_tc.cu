@@ -11,8 +11,8 @@
 // every row of a group, so one fetched stage serves all its rows; from the second level on a
 // left branch inherits its parent's score and only right branches are fetched.
 //
-// Roles (256 threads): warp 0 TMA producer, warp 1 MMA issuer + TMEM owner, warp 2 controller,
-// warps 4..7 epilogue (TMEM lane quarter = warp % 4). All roles walk the same fixed unit order
+// Roles (256 threads): warp 0 TMA producer, warps 1 and 3 MMA issuers (warp 1 owns TMEM), warp 2
+// controller, warps 4..7 epilogue (TMEM lane quarter = warp % 4). All roles walk the same fixed unit order
 // (level 1: stage-major, row-minor; later levels: row-major), synchronised by mbarriers only.
 // Every wait is bounded: on a timeout the CTA records an error code in the workspace header,
 // raises a shared abort flag, drains its own copies and leaves.
@@ -118,11 +118,15 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
     }
 }
 
-// Run by all 32 lanes of its warp, converged: the waits are warp-wide, one elected lane issues.
-__device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_smem, unsigned tmem_base) {
+// Two warps issue the chains, alternating (chain c belongs to warp c % 2): the thread that issues
+// a chain is held until the tensor core has taken it, so with one issuing warp the waits and
+// commits between chains would not overlap with the chains themselves. Both warps walk the same
+// unit order; each is run by all 32 lanes, converged: warp-wide waits, one elected lane issues.
+__device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_smem, unsigned tmem_base, int which) {
     const Geom &g = P.g;
     Ring st, sl;
     unsigned grp_par = 0, q_par = 0, jr_par[kR] = {0, 0, 0, 0};
+    unsigned chain = 0;
     const unsigned q_lo = desc_lo_sw128(q_smem, 16);
     for (;;) {
         if (!mbar_wait_w(smem_u32(&tl->jobs_ready[kR]), grp_par, tl, P.ws, 201)) return;
@@ -141,10 +145,15 @@ __device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_
                 }
                 const int n = tl->n_jobs[li];
                 for (int j = 0; j < n; j += 2) {
-                    if (!mbar_wait_w(smem_u32(&tl->full[st.idx]), st.phase, tl, P.ws, 204)) return;
-                    const unsigned a_lo = desc_lo_sw128(k_smem + st.idx * kStageBytes, 16);
                     const int r0 = level == 0 ? 0 : x, r1 = level == 0 ? R : x + 1;
-                    for (int r = r0; r < r1; ++r) {
+                    bool stage_ready = false;
+                    const unsigned a_lo = desc_lo_sw128(k_smem + st.idx * kStageBytes, 16);
+                    for (int r = r0; r < r1; ++r, ++chain, sl.advance(kSlots)) {
+                        if ((int)(chain & 1u) != which) continue;
+                        if (!stage_ready) {
+                            if (!mbar_wait_w(smem_u32(&tl->full[st.idx]), st.phase, tl, P.ws, 204)) return;
+                            stage_ready = true;
+                        }
                         if (!mbar_wait_w(smem_u32(&tl->tmem_empty[sl.idx]), sl.phase ^ 1, tl, P.ws, 205)) return;
                         tc_fence_after();
                         const unsigned d_tmem = tmem_base + sl.idx * 64;
@@ -157,11 +166,16 @@ __device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_
                                     tc_mma_bf16_split(d_tmem, a_lo + ((c * 2 * kHalfTile + k4 * 32) >> 4), kDescHi,
                                                       b_lo + ((c * kR * kHalfTile + k4 * 32) >> 4), kDescHi, kIdesc, (c | k4) != 0);
                             tc_commit(smem_u32(&tl->tmem_full[sl.idx]));
-                            if (r + 1 == r1) tc_commit(smem_u32(&tl->empty[st.idx]));
                         }
                         __syncwarp();
-                        sl.advance(kSlots);
                     }
+                    // the stage is free once both warps are done with it: the one that read it
+                    // commits behind its chains, the other (if it had none here) just arrives
+                    if (elect_one()) {
+                        if (stage_ready) tc_commit(smem_u32(&tl->empty[st.idx]));
+                        else mbar_arrive(smem_u32(&tl->empty[st.idx]));
+                    }
+                    __syncwarp();
                     st.advance(kStages);
                 }
             }
@@ -366,7 +380,7 @@ mask_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < kStages; ++i) { mbar_init(smem_u32(&tl->full[i]), 1); mbar_init(smem_u32(&tl->empty[i]), 1); }
+        for (int i = 0; i < kStages; ++i) { mbar_init(smem_u32(&tl->full[i]), 1); mbar_init(smem_u32(&tl->empty[i]), 2); }
         for (int i = 0; i < kSlots; ++i) { mbar_init(smem_u32(&tl->tmem_full[i]), 1); mbar_init(smem_u32(&tl->tmem_empty[i]), 4); }
         mbar_init(smem_u32(&tl->q_full), 1);
         for (int i = 0; i <= kR; ++i) mbar_init(smem_u32(&tl->jobs_ready[i]), 1);
@@ -386,9 +400,11 @@ mask_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     if (warp == 0) {
         if (lane == 0) producer_role(P, &tmap_q, &tmap_k, tl, q_smem, k_smem);
     } else if (warp == 1) {
-        mma_role(P, tl, q_smem, k_smem, tmem_base);
+        mma_role(P, tl, q_smem, k_smem, tmem_base, 0);
     } else if (warp == 2) {
         controller_role(P, tl, lane);
+    } else if (warp == 3) {
+        mma_role(P, tl, q_smem, k_smem, tmem_base, 1);
     } else if (warp >= 4) {
         epilogue_role(P, tl, tmem_base, warp & 3, lane);
     }

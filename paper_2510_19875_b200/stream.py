@@ -80,6 +80,8 @@ def _load():
     lib.stream_sparse_attention.argtypes = [P, vp, vp, vp, vp, ctypes.c_float, vp, vp]
     lib.stream_read_stats.restype = ctypes.c_int
     lib.stream_read_stats.argtypes = [vp, ctypes.POINTER(StreamStats), vp]
+    lib.stream_vertical_scores.restype = ctypes.c_int
+    lib.stream_vertical_scores.argtypes = [P, vp, vp, vp, vp, vp, sz, vp]
     lib.stream_check_device_status.restype = ctypes.c_int
     lib.stream_check_device_status.argtypes = [vp]
     lib.stream_host_staging_bytes.restype = sz
@@ -144,6 +146,12 @@ def stream_read_stats(workspace, stream=None) -> StreamStats:
     st = StreamStats()
     _raise(_load().stream_read_stats(_addr(workspace), ctypes.byref(st), _stream_handle(stream)))
     return st
+
+
+def stream_vertical_scores(p: StreamProblem, mask, scores, vertical_out, kurtosis_out, workspace, workspace_bytes: int,
+                           stream=None) -> None:
+    _raise(_load().stream_vertical_scores(ctypes.byref(p), _addr(mask), _addr(scores), _addr(vertical_out),
+                                          _addr(kurtosis_out), _addr(workspace), workspace_bytes, _stream_handle(stream)))
 
 
 def stream_check_device_status(stream=None) -> None:
@@ -240,3 +248,18 @@ def run_host(q_host: torch.Tensor, k_host: torch.Tensor, v_host: torch.Tensor, m
         raise ValueError("q/k/v/mask/out live on the host, staging on the device")
     p = make_problem(q_host, k_host, block_q=block_q, block_k=block_k, k_top=k_top, causal=causal, impl=impl)
     stream_run_host(p, q_host, k_host, v_host, mask_host, out_host, scale, staging, staging.numel(), stream)
+
+
+def vertical_scores(p: StreamProblem, mask: torch.Tensor, scores: torch.Tensor | None = None, stream=None):
+    """(vertical [B, H, ceil(T / block_k)], kurtosis [B, H]) of a mask, binary or weighted by ``scores``."""
+    if not mask.is_cuda or mask.dtype != torch.int32 or not mask.is_contiguous():
+        raise ValueError("mask must be a contiguous int32 CUDA tensor")
+    if scores is not None and (scores.shape != mask.shape or scores.dtype != torch.float32 or not scores.is_contiguous()):
+        raise ValueError("scores must be a contiguous float32 tensor of the mask's shape")
+    n_kb = -(-p.T // p.block_k)
+    vert = torch.empty((p.batch, p.n_q_heads, n_kb), dtype=torch.float32, device=mask.device)
+    kurt = torch.empty((p.batch, p.n_q_heads), dtype=torch.float32, device=mask.device)
+    ws = new_workspace(p, mask.device)
+    stream_vertical_scores(p, mask, scores, vert, kurt, ws, ws.numel(), stream)
+    stream_read_stats(ws, stream)
+    return vert, kurt

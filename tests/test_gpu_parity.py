@@ -272,3 +272,34 @@ def test_run_host_matches_device_calls(S):
     torch.cuda.synchronize()
     assert torch.equal(mask_host, ref.mask.cpu())
     assert torch.equal(out_host, out_ref.cpu())
+
+
+@pytest.mark.parametrize("kw", [dict(), dict(T=5000, k_top=5, n_q_heads=7, n_kv_heads=1), dict(T=3000, k_top=3, n_q_heads=6, n_kv_heads=2, batch=2)])
+def test_vertical_scores_and_kurtosis(S, kw):
+    """Column sums of the GPU mask (binary and score-weighted) and their kurtosis against the oracle
+    fed with the same mask and scores."""
+    w = wl.generate(tc_spec(**kw))
+    spec = w.spec
+    res = run_mask(S, w, want_scores=True)
+    p = S.make_problem(*w.torch_tensors("cuda")[:2], block_q=spec.block, block_k=spec.block, k_top=spec.k_top)
+    op = oracle_problem(spec)
+    mask_np = res.mask.cpu().numpy().reshape(-1, spec.k_top)
+    sc_np = res.scores.cpu().numpy().reshape(-1, spec.k_top)
+    vert, kurt = S.vertical_scores(p, res.mask)
+    ref_v, ref_k = so.vertical_scores(op, mask_np)
+    assert np.array_equal(vert.cpu().numpy().reshape(ref_v.shape), ref_v)          # counts: exact
+    np.testing.assert_allclose(kurt.cpu().numpy().reshape(-1), ref_k, rtol=1e-4)
+    wvert, wkurt = S.vertical_scores(p, res.mask, res.scores)
+    ref_wv, ref_wk = so.vertical_scores(op, mask_np, sc_np)
+    np.testing.assert_allclose(wvert.cpu().numpy().reshape(ref_wv.shape), ref_wv, rtol=1e-5, atol=1e-2)  # fp32 sums of scores ~ 50
+    np.testing.assert_allclose(wkurt.cpu().numpy().reshape(-1), ref_wk, rtol=1e-3)
+
+
+def test_vertical_scores_flags_out_of_range_entries(S):
+    w = wl.generate(tc_spec(T=1024, k_top=4))
+    q, k, _ = w.torch_tensors("cuda")
+    p = S.make_problem(q, k, block_q=64, block_k=64, k_top=4)
+    mask = torch.full((1, 4, 16, 4), 16, dtype=torch.int32, device="cuda")  # block 16 does not exist
+    with pytest.raises(S.StreamError) as e:
+        S.vertical_scores(p, mask)
+    assert e.value.status == S.STREAM_ERR_DEVICE_CHECK

@@ -350,3 +350,32 @@ def test_default_scale_is_inverse_sqrt_d():
     a = so.sparse_attention_rows(p, q, kk, v, mask)
     b = so.sparse_attention_rows(p, q, kk, v, mask, scale=0.5)
     assert (a == b).all()
+
+
+def test_vertical_scores_are_column_sums_with_library_kurtosis():
+    """Pins for the vertical scores: numpy's bincount for the sums, scipy's Pearson kurtosis for
+    the fourth-moment ratio, and a hand-worked row."""
+    from scipy import stats
+
+    p = so.OracleProblem(2, 2, 1, 96, 4, 8, 8, 3, True, "f32")
+    nq = nk = 12
+    rng = np.random.default_rng(3)
+    mask = rng.integers(-1, nk, size=(2 * 2 * nq, 3)).astype(np.int32)
+    scores = rng.standard_normal(mask.shape).astype(np.float32)
+    vert, kurt = so.vertical_scores(p, mask)
+    wvert, wkurt = so.vertical_scores(p, mask, scores)
+    for h in range(4):
+        rows = mask[h * nq:(h + 1) * nq]
+        keep = rows >= 0
+        np.testing.assert_array_equal(vert[h], np.bincount(rows[keep], minlength=nk))
+        np.testing.assert_allclose(wvert[h], np.bincount(rows[keep], weights=scores[h * nq:(h + 1) * nq][keep].astype(np.float64), minlength=nk), rtol=1e-12, atol=1e-12)
+        assert kurt[h] == pytest.approx(stats.kurtosis(vert[h], fisher=False, bias=True), rel=1e-12)
+        assert wkurt[h] == pytest.approx(stats.kurtosis(wvert[h], fisher=False, bias=True), rel=1e-12)
+    # by hand: one head, 4 key blocks, every query block keeps block 0 and itself -> v = [4, 1, 1, 1]
+    p1 = so.OracleProblem(1, 1, 1, 32, 4, 8, 8, 2, True, "f32")
+    m1 = np.array([[0, -1], [0, 1], [0, 2], [0, 3]], np.int32)
+    v1, k1 = so.vertical_scores(p1, m1)
+    assert v1.tolist() == [[4.0, 1.0, 1.0, 1.0]]
+    # mean 1.75, deviations (2.25, -.75, -.75, -.75): m2 = 1.6875, m4 = 6.64453125 -> 2.3333...
+    assert k1[0] == pytest.approx(6.64453125 / 1.6875 ** 2, rel=1e-14)
+    assert so.vertical_scores(p1, np.array([[0, -1], [1, -1], [2, -1], [3, -1]], np.int32))[1][0] == 0.0  # flat

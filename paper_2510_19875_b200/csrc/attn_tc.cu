@@ -16,7 +16,7 @@
 // output registers (o = o * alpha + O_e) one iteration later, so that the tensor core works on
 // the next logits meanwhile.
 //
-// Roles (384 threads): warp 0 TMA producer; warp 1 issues the Q K^T chains and owns TMEM; warp 3
+// Roles (384 threads): warp 0 TMA producer (converged, one elected lane issues); warp 1 issues the Q K^T chains and owns TMEM; warp 3
 // issues the P V chains (two issuing warps, because the thread that issues a chain is held until
 // the tensor core has taken it: with one warp the waits and commits between chains would not
 // overlap with the chains themselves); warp 2 copies the pairs' mask rows from global to shared
@@ -151,17 +151,23 @@ __device__ void mask_loader_role(const Params &P, Tail *tl, int lane) {
     }
 }
 
-// One thread feeds two independent streams of TMA loads, the K tiles (with each pair's Q tiles)
+// One warp feeds two independent streams of TMA loads, the K tiles (with each pair's Q tiles)
 // and the V tiles, each as far ahead as its ring of stages allows. It never blocks on one stream
-// while the other could move: every step probes its barrier without waiting.
+// while the other could move: every step probes its barrier without waiting. The warp runs
+// converged (lane 0's probe result is broadcast) and one elected lane issues.
 struct LoadStream {
     int id;            // pair being walked
     int e;             // current entry (k_top = pair exhausted), -2 = pair not opened yet
     int n_issued;      // loads issued for this pair
     Entry cur;
+    Item it;
     Ring ring, ms;
     bool q_due;        // (K stream) the pair's Q tiles still have to be requested
 };
+
+__device__ __forceinline__ bool probe_w(unsigned bar, unsigned parity) {
+    return __shfl_sync(0xffffffffu, (int)mbar_test_wait(bar, parity), 0) != 0;
+}
 
 __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUtensorMap *tk, const CUtensorMap *tv,
                               Tail *tl, unsigned q_smem, unsigned k_smem, unsigned v_smem) {
@@ -192,42 +198,48 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
         if (S.id >= P.n_items) return false;
         const int *rows = mask_rows(tl, P, S.ms.idx);
         if (S.e == -2) {  // open the pair: its mask rows must be resident
-            if (!mbar_test_wait(smem_u32(&tl->m_full[S.ms.idx]), S.ms.phase)) return false;
+            if (!probe_w(smem_u32(&tl->m_full[S.ms.idx]), S.ms.phase)) return false;
+            S.it = decode_item(P, S.id);
             S.e = next_entry(rows, P.row_stride, -1, g.k_top, &S.cur);
             S.q_due = is_k && S.e < g.k_top;  // (a pair with nothing kept: only the softmax warps act)
             S.n_issued = 0;
             return true;
         }
         if (S.e >= g.k_top && !S.q_due) {  // pair exhausted: give its mask rows back, go to the next one
-            mbar_arrive(smem_u32(&tl->m_empty[S.ms.idx]));
+            if (elect_one()) mbar_arrive(smem_u32(&tl->m_empty[S.ms.idx]));
+            __syncwarp();
             S.ms.advance(kMaskSlots);
             S.id += gridDim.x;
             S.e = -2;
             return true;
         }
-        const Item it = decode_item(P, S.id);
         if (is_k) {
             if (S.e < g.k_top && !(S.q_due && S.n_issued > 0)) {
                 // a K stage is free once the logits computed from it are complete
-                if (!mbar_test_wait(smem_u32(&tl->k_empty[S.ring.idx]), S.ring.phase ^ 1)) return false;
-                load_k_pair(k_smem + S.ring.idx * kOperand, smem_u32(&tl->k_full[S.ring.idx]), it, S.cur);
+                if (!probe_w(smem_u32(&tl->k_empty[S.ring.idx]), S.ring.phase ^ 1)) return false;
+                if (elect_one()) load_k_pair(k_smem + S.ring.idx * kOperand, smem_u32(&tl->k_full[S.ring.idx]), S.it, S.cur);
+                __syncwarp();
                 S.ring.advance(P.n_k_stages);
                 S.e = next_entry(rows, P.row_stride, S.e, g.k_top, &S.cur);
                 ++S.n_issued;
                 return true;
             }
             // Q goes behind the pair's first K tiles, which do not depend on the Q buffer
-            if (!mbar_test_wait(smem_u32(&tl->q_empty), q_par ^ 1)) return false;
+            if (!probe_w(smem_u32(&tl->q_empty), q_par ^ 1)) return false;
             q_par ^= 1;
-            const unsigned bar = smem_u32(&tl->q_full);
-            mbar_arrive_expect_tx(bar, (unsigned)kOperand);
-            tma_load_5d(q_smem, tq, bar, 0, it.qb * kBlk, it.h0, 0, it.b);  // heads h0 and h0 + 1
+            if (elect_one()) {
+                const unsigned bar = smem_u32(&tl->q_full);
+                mbar_arrive_expect_tx(bar, (unsigned)kOperand);
+                tma_load_5d(q_smem, tq, bar, 0, S.it.qb * kBlk, S.it.h0, 0, S.it.b);  // heads h0 and h0 + 1
+            }
+            __syncwarp();
             S.q_due = false;
             return true;
         }
         // a V stage is free once the product computed from it is complete
-        if (!mbar_test_wait(smem_u32(&tl->o_full[S.ring.idx]), S.ring.phase ^ 1)) return false;
-        load_v_pair(v_smem + S.ring.idx * kOperand, smem_u32(&tl->v_full[S.ring.idx]), it, S.cur);
+        if (!probe_w(smem_u32(&tl->o_full[S.ring.idx]), S.ring.phase ^ 1)) return false;
+        if (elect_one()) load_v_pair(v_smem + S.ring.idx * kOperand, smem_u32(&tl->v_full[S.ring.idx]), S.it, S.cur);
+        __syncwarp();
         S.ring.advance(kVStages);
         S.e = next_entry(rows, P.row_stride, S.e, g.k_top, &S.cur);
         return true;
@@ -238,12 +250,18 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
         if (moved_k || moved_v) {
             t_last = clock64();
         } else {
-            if (*(volatile int *)&tl->abort_flag) return;
-            if (clock64() - t_last > kWaitCycles) {
-                *(volatile int *)&tl->abort_flag = 1;
-                if (atomicCAS(&g_attn_status[0], 0u, 101u) == 0u) g_attn_status[1] = blockIdx.x;
-                return;
+            // nothing to do right now: lane 0 decides for the warp whether to go on
+            int stop = 0;
+            if ((threadIdx.x & 31) == 0) {
+                if (*(volatile int *)&tl->abort_flag) stop = 1;
+                else if (clock64() - t_last > kWaitCycles) {
+                    *(volatile int *)&tl->abort_flag = 1;
+                    if (atomicCAS(&g_attn_status[0], 0u, 101u) == 0u) g_attn_status[1] = blockIdx.x;
+                    stop = 1;
+                }
             }
+            if (__shfl_sync(0xffffffffu, stop, 0)) return;
+            __nanosleep(64);  // leave the issue slots to the softmax warps of this scheduler
         }
     }
 }
@@ -338,6 +356,12 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float y;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
+    return y;
+}
+
 // o[0..63] = o * alpha + O, O being 64 columns of this thread's lane of a TMEM buffer.
 __device__ __forceinline__ void fold_output(float *o, float alpha, unsigned taddr) {
     unsigned r[64];
@@ -412,10 +436,16 @@ __device__ void softmax_role(const Params &P, Tail *tl, unsigned char *p_ptr, un
                 n_hi = (int)max(0ll, min(lim, (long long)kBlk));
             }
             const int n_own = n_hi - part * 32, n_oth = n_hi - (part ^ 1) * 32;  // within each half
+            const bool all_keys = n_hi == kBlk;  // every block but the diagonal one and the one across T
             float mx4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
-            if (n_hi == kBlk) {
+            if (all_keys) {
 #pragma unroll
-                for (int i = 0; i < 64; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(sr[i]));
+                for (int i = 0; i < 64; i += 8) {
+                    mx4[0] = max3(mx4[0], __uint_as_float(sr[i]), __uint_as_float(sr[i + 1]));
+                    mx4[1] = max3(mx4[1], __uint_as_float(sr[i + 2]), __uint_as_float(sr[i + 3]));
+                    mx4[2] = max3(mx4[2], __uint_as_float(sr[i + 4]), __uint_as_float(sr[i + 5]));
+                    mx4[3] = max3(mx4[3], __uint_as_float(sr[i + 6]), __uint_as_float(sr[i + 7]));
+                }
             } else {
 #pragma unroll
                 for (int i = 0; i < 32; ++i) {
@@ -429,15 +459,26 @@ __device__ void softmax_role(const Params &P, Tail *tl, unsigned char *p_ptr, un
             const float alpha = m_new == m ? 1.f : fast_exp2((m - m_new) * P.scale_log2);
             float sum4[4] = {0.f, 0.f, 0.f, 0.f};
             unsigned packed[16];
+            if (all_keys) {
 #pragma unroll
-            for (int i = 0; i < 32; i += 2) {
-                float p0 = fast_exp2(fmaf(__uint_as_float(sr[i]), P.scale_log2, shift));
-                float p1 = fast_exp2(fmaf(__uint_as_float(sr[i + 1]), P.scale_log2, shift));
-                p0 = i < n_own ? p0 : 0.f;
-                p1 = i + 1 < n_own ? p1 : 0.f;
-                sum4[(i >> 1) & 3] += p0 + p1;
-                __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
-                packed[i >> 1] = *reinterpret_cast<unsigned *>(&pk);
+                for (int i = 0; i < 32; i += 2) {
+                    const float p0 = fast_exp2(fmaf(__uint_as_float(sr[i]), P.scale_log2, shift));
+                    const float p1 = fast_exp2(fmaf(__uint_as_float(sr[i + 1]), P.scale_log2, shift));
+                    sum4[(i >> 1) & 3] += p0 + p1;
+                    __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+                    packed[i >> 1] = *reinterpret_cast<unsigned *>(&pk);
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < 32; i += 2) {
+                    float p0 = fast_exp2(fmaf(__uint_as_float(sr[i]), P.scale_log2, shift));
+                    float p1 = fast_exp2(fmaf(__uint_as_float(sr[i + 1]), P.scale_log2, shift));
+                    p0 = i < n_own ? p0 : 0.f;
+                    p1 = i + 1 < n_own ? p1 : 0.f;
+                    sum4[(i >> 1) & 3] += p0 + p1;
+                    __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+                    packed[i >> 1] = *reinterpret_cast<unsigned *>(&pk);
+                }
             }
             l = l * alpha + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
             m = m_new;
@@ -531,7 +572,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     const unsigned tmem_base = tl->tmem_base;
 
     if (warp == 0) {
-        if (lane == 0) producer_role(P, &tmap_q, &tmap_k, &tmap_v, tl, q_smem, k_smem, v_smem);
+        producer_role(P, &tmap_q, &tmap_k, &tmap_v, tl, q_smem, k_smem, v_smem);
     } else if (warp == 1) {
         qk_role(P, tl, q_smem, k_smem, tmem_base);
     } else if (warp == 2) {

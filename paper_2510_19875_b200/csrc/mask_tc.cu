@@ -11,8 +11,8 @@
 // every row of a group, so one fetched stage serves all its rows; from the second level on a
 // left branch inherits its parent's score and only right branches are fetched.
 //
-// Roles (256 threads): warp 0 TMA producer, warps 1 and 3 MMA issuers (warp 1 owns TMEM), warp 2
-// controller, warps 4..7 epilogue (TMEM lane quarter = warp % 4). All roles walk the same fixed unit order
+// Roles (384 threads, the last two warps idle): warp 0 TMA producer, warps 1, 3, 8, 9 MMA issuers
+// (warp 1 owns TMEM), warp 2 controller, warps 4..7 epilogue (TMEM lane quarter = warp % 4). All roles walk the same fixed unit order
 // (level 1: stage-major, row-minor; later levels: row-major), synchronised by mbarriers only.
 // Every wait is bounded: on a timeout the CTA records an error code in the workspace header,
 // raises a shared abort flag, drains its own copies and leaves.
@@ -25,7 +25,8 @@ namespace {
 
 using namespace tc;
 
-constexpr int kThreads = 256;
+constexpr int kThreads = 384;
+constexpr int kMmaWarps = 4;   // warps 1, 3, 8, 9 issue the chains in turn
 constexpr int kR = 4;          // rows (query heads) per group
 constexpr int kStages = 4;     // K-pair stages
 constexpr int kSlots = 8;      // TMEM accumulator slots of 64 fp32 columns
@@ -76,41 +77,50 @@ struct Params {
 // ----------------------------------------------------------------------------------------------
 // Roles
 // ----------------------------------------------------------------------------------------------
+// Run by all 32 lanes of warp 0, converged (warp-wide waits, one elected lane issues): a single
+// diverged lane issues TMA copies several times more slowly.
 __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUtensorMap *tk, Tail *tl, unsigned q_smem,
                               unsigned k_smem) {
     const Geom &g = P.g;
     Ring st;
     unsigned grp_par = 0, jr_par[kR] = {0, 0, 0, 0};
     for (;;) {
-        if (!mbar_wait(smem_u32(&tl->jobs_ready[kR]), grp_par, tl, P.ws, 101)) return;
+        if (!mbar_wait_w(smem_u32(&tl->jobs_ready[kR]), grp_par, tl, P.ws, 101)) return;
         grp_par ^= 1;
         if (tl->grp_id < 0) return;
         const int b = tl->grp_b, kvh = tl->grp_kvh, qb = tl->grp_qb, h0 = tl->grp_h0, R = tl->grp_R;
         // Q tiles of the group's rows (previous group's MMAs are all complete by now)
-        mbar_arrive_expect_tx(smem_u32(&tl->q_full), (unsigned)(R * 2 * kHalfTile));
-        for (int r = 0; r < R; ++r)
-            for (int c = 0; c < 2; ++c)
-                tma_load_4d(q_smem + (c * kR + r) * kHalfTile, tq, smem_u32(&tl->q_full), c * 64, qb * kBlk, h0 + r, b);
+        if (elect_one()) {
+            mbar_arrive_expect_tx(smem_u32(&tl->q_full), (unsigned)(R * 2 * kHalfTile));
+            for (int r = 0; r < R; ++r)
+                for (int c = 0; c < 2; ++c)
+                    tma_load_4d(q_smem + (c * kR + r) * kHalfTile, tq, smem_u32(&tl->q_full), c * 64, qb * kBlk, h0 + r, b);
+        }
+        __syncwarp();
         for (int level = 0; level < g.levels; ++level) {
             const int lists = level == 0 ? 1 : R;
             for (int x = 0; x < lists; ++x) {
                 const int li = level == 0 ? kR : x;
                 if (level > 0) {
-                    if (!mbar_wait(smem_u32(&tl->jobs_ready[x]), jr_par[x], tl, P.ws, 102)) return;
+                    if (!mbar_wait_w(smem_u32(&tl->jobs_ready[x]), jr_par[x], tl, P.ws, 102)) return;
                     jr_par[x] ^= 1;
                 }
                 const int n = tl->n_jobs[li];
                 for (int j = 0; j < n; j += 2) {
-                    if (!mbar_wait(smem_u32(&tl->empty[st.idx]), st.phase ^ 1, tl, P.ws, 103)) return;
+                    if (!mbar_wait_w(smem_u32(&tl->empty[st.idx]), st.phase ^ 1, tl, P.ws, 103)) return;
                     const int two = (j + 1 < n);
-                    const unsigned bar = smem_u32(&tl->full[st.idx]);
-                    const unsigned dst = k_smem + st.idx * kStageBytes;
-                    mbar_arrive_expect_tx(bar, (unsigned)((two ? 4 : 2) * kHalfTile));
-                    for (int t = 0; t <= two; ++t) {
-                        const int blk = tl->jobs_blk[li][j + t];
-                        for (int c = 0; c < 2; ++c)
-                            tma_load_4d(dst + (c * 2 + t) * kHalfTile, tk, bar, c * 64, blk * kBlk, kvh, b);
+                    const int blk0 = tl->jobs_blk[li][j], blk1 = two ? tl->jobs_blk[li][j + 1] : 0;
+                    if (elect_one()) {
+                        const unsigned bar = smem_u32(&tl->full[st.idx]);
+                        const unsigned dst = k_smem + st.idx * kStageBytes;
+                        mbar_arrive_expect_tx(bar, (unsigned)((two ? 4 : 2) * kHalfTile));
+#pragma unroll
+                        for (int c = 0; c < 2; ++c) {
+                            tma_load_4d(dst + c * 2 * kHalfTile, tk, bar, c * 64, blk0 * kBlk, kvh, b);
+                            if (two) tma_load_4d(dst + (c * 2 + 1) * kHalfTile, tk, bar, c * 64, blk1 * kBlk, kvh, b);
+                        }
                     }
+                    __syncwarp();
                     st.advance(kStages);
                 }
             }
@@ -118,10 +128,11 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
     }
 }
 
-// Two warps issue the chains, alternating (chain c belongs to warp c % 2): the thread that issues
-// a chain is held until the tensor core has taken it, so with one issuing warp the waits and
-// commits between chains would not overlap with the chains themselves. Both warps walk the same
-// unit order; each is run by all 32 lanes, converged: warp-wide waits, one elected lane issues.
+// kMmaWarps warps issue the chains in turn (chain c belongs to warp c % kMmaWarps): the waits,
+// commits and bookkeeping between two chains of one warp take several times longer than the
+// tensor core needs for a chain, so one issuing warp would leave it idle most of the time. All
+// issuing warps walk the same unit order; each is run by all 32 lanes, converged: warp-wide
+// waits, one elected lane issues.
 __device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_smem, unsigned tmem_base, int which) {
     const Geom &g = P.g;
     Ring st, sl;
@@ -149,7 +160,7 @@ __device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_
                     bool stage_ready = false;
                     const unsigned a_lo = desc_lo_sw128(k_smem + st.idx * kStageBytes, 16);
                     for (int r = r0; r < r1; ++r, ++chain, sl.advance(kSlots)) {
-                        if ((int)(chain & 1u) != which) continue;
+                        if ((int)(chain % kMmaWarps) != which) continue;
                         if (!stage_ready) {
                             if (!mbar_wait_w(smem_u32(&tl->full[st.idx]), st.phase, tl, P.ws, 204)) return;
                             stage_ready = true;
@@ -169,8 +180,8 @@ __device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_
                         }
                         __syncwarp();
                     }
-                    // the stage is free once both warps are done with it: the one that read it
-                    // commits behind its chains, the other (if it had none here) just arrives
+                    // the stage is free once every issuing warp is done with it: those that read it
+                    // commit behind their chains, the others just arrive
                     if (elect_one()) {
                         if (stage_ready) tc_commit(smem_u32(&tl->empty[st.idx]));
                         else mbar_arrive(smem_u32(&tl->empty[st.idx]));
@@ -380,7 +391,7 @@ mask_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < kStages; ++i) { mbar_init(smem_u32(&tl->full[i]), 1); mbar_init(smem_u32(&tl->empty[i]), 2); }
+        for (int i = 0; i < kStages; ++i) { mbar_init(smem_u32(&tl->full[i]), 1); mbar_init(smem_u32(&tl->empty[i]), kMmaWarps); }
         for (int i = 0; i < kSlots; ++i) { mbar_init(smem_u32(&tl->tmem_full[i]), 1); mbar_init(smem_u32(&tl->tmem_empty[i]), 4); }
         mbar_init(smem_u32(&tl->q_full), 1);
         for (int i = 0; i <= kR; ++i) mbar_init(smem_u32(&tl->jobs_ready[i]), 1);
@@ -398,14 +409,16 @@ mask_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     const unsigned tmem_base = tl->tmem_base;
 
     if (warp == 0) {
-        if (lane == 0) producer_role(P, &tmap_q, &tmap_k, tl, q_smem, k_smem);
+        producer_role(P, &tmap_q, &tmap_k, tl, q_smem, k_smem);
     } else if (warp == 1) {
         mma_role(P, tl, q_smem, k_smem, tmem_base, 0);
     } else if (warp == 2) {
         controller_role(P, tl, lane);
     } else if (warp == 3) {
         mma_role(P, tl, q_smem, k_smem, tmem_base, 1);
-    } else if (warp >= 4) {
+    } else if (warp == 8 || warp == 9) {
+        mma_role(P, tl, q_smem, k_smem, tmem_base, warp - 6);
+    } else if (warp >= 4 && warp < 8) {
         epilogue_role(P, tl, tmem_base, warp & 3, lane);
     }
     __syncwarp();

@@ -198,14 +198,19 @@ size_t stream_host_staging_bytes(const stream_problem *p);
 /*
  * The whole path from HOST memory: copy Q, K, V to the device, build the mask, run the sparse
  * attention, copy mask and output back. Strides in *p describe the HOST tensors, which must be
- * dense ([batch, heads, T, d] contiguous); pinned host memory makes the copies asynchronous.
+ * dense ([batch, heads, T, d] contiguous). The work is cut into one chunk per (batch entry, kv
+ * head) - nothing else depends on a chunk - and chunk c + 1's copy in, chunk c's kernels and
+ * chunk c - 1's copy out run at the same time: the copies on two streams the library creates
+ * once per device at the first call (with a few events; kept until the process ends), the
+ * kernels on cuda_stream. Pinned host memory is what makes the copies asynchronous.
  *
  *   q_host, k_host, v_host   HOST, read only
  *   mask_host                HOST int32 [batch, n_q_heads, ceil(T/block_q), k_top]
  *   out_host                 HOST, dtype of the problem, [batch, n_q_heads, T, d]
  *   staging                  DEVICE, 256-byte aligned, >= stream_host_staging_bytes(p)
- * Returns after everything is enqueued on cuda_stream; the host buffers are valid once the
- * stream has been synchronised.
+ * Everything is ordered after what cuda_stream already holds, and cuda_stream is made to wait
+ * for the last copy out: the host buffers are valid once cuda_stream has been synchronised. Two
+ * calls that share a device must not overlap in time (they share the internal streams' events).
  */
 stream_status stream_run_host(const stream_problem *p, const void *q_host, const void *k_host, const void *v_host,
                               int32_t *mask_host, void *out_host, float scale, void *staging,

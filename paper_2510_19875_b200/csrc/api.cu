@@ -2,6 +2,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 
 #include "common.cuh"
 
@@ -84,6 +85,39 @@ StagingLayout staging_layout(const stream_problem *p, const Geom &g) {
     s.q = 0; s.k = s.q + align256(qb); s.v = s.k + align256(kb); s.mask = s.v + align256(kb);
     s.out = s.mask + align256(mb); s.ws = s.out + align256(qb); s.total = s.ws + sizeof(WorkspaceHeader);
     return s;
+}
+
+// Streams and events behind stream_run_host, made once per device and kept for the life of the
+// process: one stream for the copies in, one for the copies out (the kernels run on the
+// caller's stream), and a few events to chain the three.
+constexpr int kPipeEvents = 4;
+struct HostPipe {
+    bool ready = false;
+    cudaStream_t in = nullptr, out = nullptr;
+    cudaEvent_t start = nullptr, finish = nullptr, in_done[kPipeEvents] = {}, comp_done[kPipeEvents] = {};
+};
+constexpr int kMaxPipeDevices = 64;
+std::mutex g_pipe_mu;
+HostPipe g_pipes[kMaxPipeDevices];
+
+stream_status host_pipe_for_current_device(HostPipe **out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    if (dev < 0 || dev >= kMaxPipeDevices) { set_error("device ordinal %d outside 0..%d", dev, kMaxPipeDevices - 1); return STREAM_ERR_UNSUPPORTED; }
+    std::lock_guard<std::mutex> lock(g_pipe_mu);
+    HostPipe &hp = g_pipes[dev];
+    if (!hp.ready) {
+        if ((e = cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e, "cudaStreamCreate");
+        if ((e = cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e, "cudaStreamCreate");
+        cudaEvent_t *evs[2 + 2 * kPipeEvents] = {&hp.start, &hp.finish};
+        for (int i = 0; i < kPipeEvents; ++i) { evs[2 + i] = &hp.in_done[i]; evs[2 + kPipeEvents + i] = &hp.comp_done[i]; }
+        for (cudaEvent_t *ev : evs)
+            if ((e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e, "cudaEventCreate");
+        hp.ready = true;
+    }
+    *out = &hp;
+    return STREAM_OK;
 }
 
 bool dense_layout(const stream_problem *p) {
@@ -212,23 +246,48 @@ stream_status stream_run_host(const stream_problem *p, const void *q_host, const
         set_error("staging must be a 256-byte aligned device buffer of at least %zu bytes", s.total);
         return STREAM_ERR_WORKSPACE;
     }
+    HostPipe *hp = nullptr;
+    rc = host_pipe_for_current_device(&hp);
+    if (rc != STREAM_OK) return rc;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     char *base = (char *)staging;
-    size_t e = elem_size(p->dtype);
-    size_t qb = (size_t)g.batch * g.H * g.T * g.d * e, kb = (size_t)g.batch * g.G * g.T * g.d * e;
-    size_t mb = (size_t)g.batch * g.H * g.n_qb * g.k_top * sizeof(int32_t);
+    const size_t e = elem_size(p->dtype);
+    // One chunk = one kv head of one batch entry with its query heads: nothing else depends on it,
+    // so its copy in, its two kernels and its copy out can overlap with the neighbours'.
+    const size_t q_chunk = (size_t)g.hpg * g.T * g.d * e, kv_chunk = (size_t)g.T * g.d * e;
+    const size_t m_chunk = (size_t)g.hpg * g.n_qb * g.k_top * sizeof(int32_t);
+    stream_problem sub = *p;
+    sub.batch = 1; sub.n_q_heads = g.hpg; sub.n_kv_heads = 1;
     cudaError_t ce;
-    if ((ce = cudaMemcpyAsync(base + s.q, q_host, qb, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(ce, "H2D q");
-    if ((ce = cudaMemcpyAsync(base + s.k, k_host, kb, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(ce, "H2D k");
-    if ((ce = cudaMemcpyAsync(base + s.v, v_host, kb, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(ce, "H2D v");
-    rc = stream_build_mask(p, base + s.q, base + s.k, (int32_t *)(base + s.mask), nullptr, base + s.ws,
-                           sizeof(WorkspaceHeader), cuda_stream);
-    if (rc != STREAM_OK) return rc;
-    rc = stream_sparse_attention(p, base + s.q, base + s.k, base + s.v, (const int32_t *)(base + s.mask), scale,
-                                 base + s.out, cuda_stream);
-    if (rc != STREAM_OK) return rc;
-    if ((ce = cudaMemcpyAsync(mask_host, base + s.mask, mb, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(ce, "D2H mask");
-    if ((ce = cudaMemcpyAsync(out_host, base + s.out, qb, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(ce, "D2H out");
+#define STREAM_TRY(call, what) do { if ((ce = (call)) != cudaSuccess) return cuda_fail(ce, what); } while (0)
+    // the internal streams start after everything already enqueued on the caller's stream
+    STREAM_TRY(cudaEventRecord(hp->start, st), "cudaEventRecord");
+    STREAM_TRY(cudaStreamWaitEvent(hp->in, hp->start, 0), "cudaStreamWaitEvent");
+    STREAM_TRY(cudaStreamWaitEvent(hp->out, hp->start, 0), "cudaStreamWaitEvent");
+    const int n_chunks = g.batch * g.G;
+    for (int c = 0; c < n_chunks; ++c) {
+        const size_t qo = (size_t)c * q_chunk, ko = (size_t)c * kv_chunk, mo = (size_t)c * m_chunk;
+        cudaEvent_t in_done = hp->in_done[c % kPipeEvents], comp_done = hp->comp_done[c % kPipeEvents];
+        STREAM_TRY(cudaMemcpyAsync(base + s.q + qo, (const char *)q_host + qo, q_chunk, cudaMemcpyHostToDevice, hp->in), "H2D q");
+        STREAM_TRY(cudaMemcpyAsync(base + s.k + ko, (const char *)k_host + ko, kv_chunk, cudaMemcpyHostToDevice, hp->in), "H2D k");
+        STREAM_TRY(cudaMemcpyAsync(base + s.v + ko, (const char *)v_host + ko, kv_chunk, cudaMemcpyHostToDevice, hp->in), "H2D v");
+        STREAM_TRY(cudaEventRecord(in_done, hp->in), "cudaEventRecord");
+        STREAM_TRY(cudaStreamWaitEvent(st, in_done, 0), "cudaStreamWaitEvent");
+        rc = stream_build_mask(&sub, base + s.q + qo, base + s.k + ko, (int32_t *)(base + s.mask + mo), nullptr, base + s.ws,
+                               sizeof(WorkspaceHeader), cuda_stream);
+        if (rc != STREAM_OK) return rc;
+        rc = stream_sparse_attention(&sub, base + s.q + qo, base + s.k + ko, base + s.v + ko,
+                                     (const int32_t *)(base + s.mask + mo), scale, base + s.out + qo, cuda_stream);
+        if (rc != STREAM_OK) return rc;
+        STREAM_TRY(cudaEventRecord(comp_done, st), "cudaEventRecord");
+        STREAM_TRY(cudaStreamWaitEvent(hp->out, comp_done, 0), "cudaStreamWaitEvent");
+        STREAM_TRY(cudaMemcpyAsync((char *)mask_host + mo, base + s.mask + mo, m_chunk, cudaMemcpyDeviceToHost, hp->out), "D2H mask");
+        STREAM_TRY(cudaMemcpyAsync((char *)out_host + qo, base + s.out + qo, q_chunk, cudaMemcpyDeviceToHost, hp->out), "D2H out");
+    }
+    // the caller's stream is done when the last copy out is
+    STREAM_TRY(cudaEventRecord(hp->finish, hp->out), "cudaEventRecord");
+    STREAM_TRY(cudaStreamWaitEvent(st, hp->finish, 0), "cudaStreamWaitEvent");
+#undef STREAM_TRY
     return STREAM_OK;
 }
 

@@ -45,6 +45,9 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="target CPU time of the oracle sample")
+    ap.add_argument("--sweep", action="store_true",
+                    help="instead of the benchmark line: time and peak memory of the sweep workload at every context "
+                         "length, with the T log T / T fits (one JSON object)")
     return ap.parse_args()
 
 
@@ -386,9 +389,79 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def fit_r2(x, y, through_origin):
+    """Least-squares line y ~ a x (+ b); returns (a, b, R^2)."""
+    import numpy as np
+
+    x, y = np.asarray(x, float), np.asarray(y, float)
+    if through_origin:
+        a, b = float((x * y).sum() / (x * x).sum()), 0.0
+    else:
+        a, b = (float(v) for v in np.polyfit(x, y, 1))
+    ss_res, ss_tot = float(((y - (a * x + b)) ** 2).sum()), float(((y - y.mean()) ** 2).sum())
+    return a, b, 1.0 - ss_res / ss_tot
+
+
+def run_sweep(args):
+    """Scaling of the path with the context length (the paper's complexity ablation, App. A.3): time of
+    both kernels and peak device memory at every T of the sweep workload, and the fits time ~ T (L + 1)
+    (L = levels of the hierarchy, about log2(T / (block k))) and memory ~ T."""
+    import math
+
+    import torch
+
+    from paper_2510_19875_b200 import stream as S
+    from paper_2510_19875_b200 import workloads as wl
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    rows = []
+    for T in wl.SWEEP_T:
+        spec = wl.SPECS["sweep"].scaled(T=T)
+        w = wl.generate(spec)
+        torch.cuda.empty_cache()
+        torch.cuda.reset_peak_memory_stats()
+        q, k, v = w.torch_tensors(dev)
+        kw = dict(block_q=spec.block, block_k=spec.block, k_top=spec.k_top)
+        p = S.make_problem(q, k, **kw)
+        mask = torch.empty((spec.batch, spec.n_q_heads, S.n_query_blocks(p), spec.k_top), dtype=torch.int32, device=dev)
+        out = torch.empty_like(q)
+        ws = S.new_workspace(p, dev)
+        stream = torch.cuda.current_stream()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        best = [float("inf"), float("inf")]
+        for it in range(5):
+            ev[0].record()
+            S.stream_build_mask(p, q, k, mask, None, ws, ws.numel(), stream)
+            ev[1].record()
+            S.stream_sparse_attention(p, q, k, v, mask, 0.0, out, stream)
+            ev[2].record()
+            torch.cuda.synchronize()
+            if it >= 2:
+                best = [min(best[0], ev[0].elapsed_time(ev[1])), min(best[1], ev[1].elapsed_time(ev[2]))]
+        tiles = int(S.stream_read_stats(ws, stream).tiles_scored)
+        n_kb = -(-T // spec.block)
+        levels = max(1, math.ceil(math.log2(max(1, -(-n_kb // spec.k_top))))) if n_kb > 1 else 0
+        rows.append({"T": T, "levels": levels, "mask_ms": best[0], "attention_ms": best[1], "tiles_scored": tiles,
+                     "peak_device_bytes": int(torch.cuda.max_memory_allocated()),
+                     "input_output_bytes": int((2 * q.numel() + 2 * k.numel()) * q.element_size() + mask.numel() * 4),
+                     "workspace_bytes": int(ws.numel())})
+        del q, k, v, out, mask, w
+    Ts = [r["T"] for r in rows]
+    a, _, r2_time = fit_r2([r["T"] * (r["levels"] + 1) for r in rows], [r["mask_ms"] for r in rows], True)
+    a_lin, _, r2_lin = fit_r2(Ts, [r["mask_ms"] for r in rows], True)
+    m_a, m_b, r2_mem = fit_r2(Ts, [r["peak_device_bytes"] for r in rows], False)
+    print(json.dumps({"workload": "sweep", "rows": rows,
+                      "fit_mask_time_vs_T_levels": {"ms_per_token_level": a, "r2": r2_time},
+                      "fit_mask_time_vs_T": {"ms_per_token": a_lin, "r2": r2_lin},
+                      "fit_peak_memory_vs_T": {"bytes_per_token": m_a, "offset_bytes": m_b, "r2": r2_mem}}))
+
+
 def main():
     args = parse_args()
-    if args.impl == "reference":
+    if args.sweep:
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

@@ -104,13 +104,16 @@ struct Item {
 __device__ __forceinline__ Item decode_item(const Params &P, int id) {
     const Geom &g = P.g;
     Item it;
-    const int per_qb = g.batch * g.G * P.n_pairs;
-    it.qb = g.n_qb - 1 - id / per_qb;  // late query blocks (most kept blocks under a causal mask) first
-    int rem = id % per_qb;
+    // kv head by kv head, so that the K and V tiles in flight belong to one head at a time (64 MiB
+    // at T = 131072: they stay in L2); within a head late query blocks (most kept blocks under a
+    // causal mask) first
+    const int per_head = g.n_qb * P.n_pairs;
+    const int bh = id / per_head;
+    const int rem = id % per_head;
+    it.qb = g.n_qb - 1 - rem / P.n_pairs;
     const int pair = rem % P.n_pairs;
-    rem /= P.n_pairs;
-    it.kvh = rem % g.G;
-    it.b = rem / g.G;
+    it.kvh = bh % g.G;
+    it.b = bh / g.G;
     it.h0 = it.kvh * g.hpg + pair * 2;
     it.R = min(2, g.hpg - pair * 2);
     return it;

@@ -30,6 +30,19 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
     return ok != 0;
 }
 
+// The same, but the hardware may keep the thread suspended for up to `ns` nanoseconds while the
+// phase is incomplete, instead of returning at once: far fewer shared-memory transactions than
+// polling, and the shared-memory port is what these kernels run against.
+__device__ __forceinline__ bool mbar_try_wait_suspend(unsigned bar, unsigned parity, unsigned ns) {
+    unsigned ok;
+    asm volatile(
+        "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\nselp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(ns)
+        : "memory");
+    return ok != 0;
+}
+
 // Non-blocking probe of an mbarrier phase.
 __device__ __forceinline__ bool mbar_test_wait(unsigned bar, unsigned parity) {
     unsigned ok;
@@ -48,7 +61,7 @@ static __device__ __noinline__ bool mbar_wait_slow(unsigned bar, unsigned parity
                                                    unsigned *err_info, unsigned code) {
     const long long t0 = clock64();
     for (;;) {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (mbar_try_wait_suspend(bar, parity, 4000u)) return true;
         if (*(volatile int *)abort_flag) return false;
         if (clock64() - t0 > kWaitCycles) {
             *(volatile int *)abort_flag = 1;
@@ -143,6 +156,16 @@ __device__ __forceinline__ void tmem_ld_32x32_issue(unsigned taddr, unsigned *r)
           "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
           "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
           "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+// The same for 16 consecutive columns.
+__device__ __forceinline__ void tmem_ld_32x16_issue(unsigned taddr, unsigned *r) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(taddr)
         : "memory");
 }

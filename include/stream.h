@@ -174,6 +174,22 @@ stream_status stream_vertical_scores(const stream_problem *p, const int32_t *mas
                                      float *kurtosis_out, void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Mask subtraction (Section 4.2 of the paper, "Exploring Information Flow": the sparse masks
+ * found with a smaller budget k are subtracted from those found with a larger one; what is left,
+ * weighted by the larger mask's block scores, are the connections only the larger budget keeps).
+ * Row by row: the entries of mask_a that are >= 0 and do not occur in the same row of mask_b, in
+ * mask_a's order, then -1 padding (their scores, then -inf padding).
+ *
+ *   n_rows           rows of both masks (batch * n_q_heads * query blocks)
+ *   mask_a, mask_b   device int32 [n_rows, k_a] and [n_rows, k_b], 1 <= k_a, k_b <= 1024; any order
+ *   scores_a         device float32 [n_rows, k_a] or NULL
+ *   diff_out         device int32 [n_rows, k_a]; overwritten; must not alias the inputs
+ *   diff_scores_out  device float32 [n_rows, k_a] or NULL (needs scores_a)
+ */
+stream_status stream_mask_difference(int64_t n_rows, int32_t k_a, const int32_t *mask_a, const float *scores_a, int32_t k_b,
+                                     const int32_t *mask_b, int32_t *diff_out, float *diff_scores_out, void *cuda_stream);
+
+/*
  * Synchronous read-back of the counters left by the last stream_build_mask that used this
  * workspace. Waits for `cuda_stream` to drain, copies the header to *out (HOST pointer) and
  * returns STREAM_ERR_DEVICE_CHECK if the kernel recorded a failed device-side check (a bounded

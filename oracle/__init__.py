@@ -3,6 +3,7 @@ from .stream_oracle import (  # noqa: F401
     OracleProblem,
     build,
     build_mask_rows,
+    mask_difference,
     num_query_blocks,
     num_rows,
     sparse_attention_rows,

@@ -365,3 +365,34 @@ int so_vertical_scores(const so_problem *p, const int32_t *mask, const float *sc
     }
     return 0;
 }
+
+/*
+ * Mask subtraction (Section 4.2, "Exploring Information Flow": the masks found with a smaller k
+ * are subtracted from those found with a larger k, and what is left - weighted by the larger
+ * mask's block scores - are the connections that only the larger budget keeps).
+ *   mask_a [n_rows, k_a], score_a same shape or NULL; mask_b [n_rows, k_b]
+ *   diff_out [n_rows, k_a]: the entries of row a (in their order) that are >= 0 and do not occur
+ *   in row b, then -1 padding; diff_score_out (if score_a): their scores, then -inf padding.
+ */
+int so_mask_difference(int64_t n_rows, int32_t k_a, const int32_t *mask_a, const float *score_a, int32_t k_b,
+                       const int32_t *mask_b, int32_t *diff_out, float *diff_score_out) {
+    if (n_rows < 0 || k_a < 1 || k_b < 1 || !mask_a || !mask_b || !diff_out) return -2;
+    for (int64_t i = 0; i < n_rows; ++i) {
+        const int32_t *a = mask_a + i * k_a, *b = mask_b + i * k_b;
+        int32_t n = 0;
+        for (int32_t j = 0; j < k_a; ++j) {
+            if (a[j] < 0) continue;
+            int found = 0;
+            for (int32_t u = 0; u < k_b; ++u) if (b[u] == a[j]) found = 1;
+            if (found) continue;
+            diff_out[i * k_a + n] = a[j];
+            if (score_a && diff_score_out) diff_score_out[i * k_a + n] = score_a[i * k_a + j];
+            ++n;
+        }
+        for (; n < k_a; ++n) {
+            diff_out[i * k_a + n] = -1;
+            if (score_a && diff_score_out) diff_score_out[i * k_a + n] = -INFINITY;
+        }
+    }
+    return 0;
+}

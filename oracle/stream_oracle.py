@@ -104,6 +104,8 @@ def _load():
         lib.so_sparse_attention_rows.restype = ctypes.c_int
         lib.so_sparse_attention_rows.argtypes = [ctypes.POINTER(_CProblem), vp, vp, vp, i64p, ctypes.c_int64,
                                                  vp, ctypes.c_double, vp]
+        lib.so_mask_difference.restype = ctypes.c_int
+        lib.so_mask_difference.argtypes = [ctypes.c_int64, ctypes.c_int32, vp, vp, ctypes.c_int32, vp, vp, vp]
         lib.so_vertical_scores.restype = ctypes.c_int
         lib.so_vertical_scores.argtypes = [ctypes.POINTER(_CProblem), vp, vp, vp, vp]
         _lib = lib
@@ -204,3 +206,21 @@ def vertical_scores(p: OracleProblem, mask: np.ndarray, scores: np.ndarray | Non
     if rc:
         raise RuntimeError(f"so_vertical_scores failed with {rc}")
     return vert, kurt
+
+
+def mask_difference(mask_a: np.ndarray, mask_b: np.ndarray, scores_a: np.ndarray | None = None):
+    """Row-wise ``mask_a`` minus ``mask_b`` ([n, k_a], [n, k_b]); returns (diff [n, k_a], scores or None)."""
+    lib = _load()
+    mask_a = np.ascontiguousarray(mask_a, dtype=np.int32)
+    mask_b = np.ascontiguousarray(mask_b, dtype=np.int32)
+    if mask_a.ndim != 2 or mask_b.ndim != 2 or mask_a.shape[0] != mask_b.shape[0]:
+        raise ValueError("masks must be [n, k_a] and [n, k_b]")
+    if scores_a is not None:
+        scores_a = np.ascontiguousarray(scores_a, dtype=np.float32)
+    diff = np.empty_like(mask_a)
+    dsc = np.empty(mask_a.shape, np.float32) if scores_a is not None else None
+    rc = lib.so_mask_difference(mask_a.shape[0], mask_a.shape[1], _ptr(mask_a), _ptr(scores_a), mask_b.shape[1],
+                                _ptr(mask_b), _ptr(diff), _ptr(dsc))
+    if rc:
+        raise RuntimeError(f"so_mask_difference failed with {rc}")
+    return diff, dsc

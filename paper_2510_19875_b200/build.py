@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libstream.so")
-SOURCES = ["api.cu", "mask_generic.cu", "attn_generic.cu", "mask_tc.cu", "attn_tc.cu", "static_scratch.cu", "vertical.cu"]
+SOURCES = ["api.cu", "mask_generic.cu", "attn_generic.cu", "mask_tc.cu", "attn_tc.cu", "static_scratch.cu", "vertical.cu", "mask_diff.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "-shared", "-Xptxas", "-v",

@@ -216,6 +216,17 @@ stream_status stream_vertical_scores(const stream_problem *p, const int32_t *mas
     return launch_vertical(g, mask, scores, vertical_out, kurtosis_out, &ws->error, st);
 }
 
+stream_status stream_mask_difference(int64_t n_rows, int32_t k_a, const int32_t *mask_a, const float *scores_a, int32_t k_b,
+                                     const int32_t *mask_b, int32_t *diff_out, float *diff_scores_out, void *cuda_stream) {
+    if (n_rows < 0 || k_a < 1 || k_b < 1 || k_a > kMaxKTop || k_b > kMaxKTop) {
+        set_error("need n_rows >= 0 and 1 <= k_a, k_b <= %d", kMaxKTop);
+        return STREAM_ERR_INVALID_ARG;
+    }
+    if (mask_a == nullptr || mask_b == nullptr || diff_out == nullptr) { set_error("mask_a, mask_b and diff_out must not be NULL"); return STREAM_ERR_INVALID_ARG; }
+    if (diff_scores_out != nullptr && scores_a == nullptr) { set_error("diff_scores_out needs scores_a"); return STREAM_ERR_INVALID_ARG; }
+    return launch_mask_diff(n_rows, k_a, mask_a, scores_a, k_b, mask_b, diff_out, diff_scores_out, (cudaStream_t)cuda_stream);
+}
+
 stream_status stream_check_device_status(void *cuda_stream) {
     unsigned int words[2] = {0, 0};
     stream_status rc = read_attn_status(words, (cudaStream_t)cuda_stream);

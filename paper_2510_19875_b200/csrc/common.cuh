@@ -50,6 +50,8 @@ stream_status launch_attn_tc(const Geom &g, const void *q, const void *k, const 
 // bad_flag: device word that gets bit 0 set if a mask entry is >= the number of key blocks.
 stream_status launch_vertical(const Geom &g, const int32_t *mask, const float *score, float *vertical, float *kurtosis,
                               unsigned int *bad_flag, cudaStream_t st);
+stream_status launch_mask_diff(long long n_rows, int k_a, const int32_t *mask_a, const float *score_a, int k_b,
+                               const int32_t *mask_b, int32_t *diff, float *diff_score, cudaStream_t st);
 // Drains `st` and copies the tensor-core attention kernel's status words (code, block) to out.
 stream_status read_attn_status(unsigned int out[2], cudaStream_t st);
 

@@ -82,6 +82,8 @@ def _load():
     lib.stream_read_stats.argtypes = [vp, ctypes.POINTER(StreamStats), vp]
     lib.stream_vertical_scores.restype = ctypes.c_int
     lib.stream_vertical_scores.argtypes = [P, vp, vp, vp, vp, vp, sz, vp]
+    lib.stream_mask_difference.restype = ctypes.c_int
+    lib.stream_mask_difference.argtypes = [ctypes.c_int64, ctypes.c_int32, vp, vp, ctypes.c_int32, vp, vp, vp, vp]
     lib.stream_check_device_status.restype = ctypes.c_int
     lib.stream_check_device_status.argtypes = [vp]
     lib.stream_host_staging_bytes.restype = sz
@@ -152,6 +154,11 @@ def stream_vertical_scores(p: StreamProblem, mask, scores, vertical_out, kurtosi
                            stream=None) -> None:
     _raise(_load().stream_vertical_scores(ctypes.byref(p), _addr(mask), _addr(scores), _addr(vertical_out),
                                           _addr(kurtosis_out), _addr(workspace), workspace_bytes, _stream_handle(stream)))
+
+
+def stream_mask_difference(n_rows: int, k_a: int, mask_a, scores_a, k_b: int, mask_b, diff_out, diff_scores_out, stream=None) -> None:
+    _raise(_load().stream_mask_difference(n_rows, k_a, _addr(mask_a), _addr(scores_a), k_b, _addr(mask_b), _addr(diff_out),
+                                          _addr(diff_scores_out), _stream_handle(stream)))
 
 
 def stream_check_device_status(stream=None) -> None:
@@ -263,3 +270,28 @@ def vertical_scores(p: StreamProblem, mask: torch.Tensor, scores: torch.Tensor |
     stream_vertical_scores(p, mask, scores, vert, kurt, ws, ws.numel(), stream)
     stream_read_stats(ws, stream)
     return vert, kurt
+
+
+def mask_difference(mask_a: torch.Tensor, mask_b: torch.Tensor, scores_a: torch.Tensor | None = None, stream=None):
+    """Row-wise ``mask_a`` minus ``mask_b`` (same leading shape, last dims k_a and k_b); returns (diff, scores or None)."""
+    if mask_a.shape[:-1] != mask_b.shape[:-1] or mask_a.dtype != torch.int32 or mask_b.dtype != torch.int32:
+        raise ValueError("masks must be int32 with the same leading shape")
+    if not (mask_a.is_cuda and mask_b.is_cuda and mask_a.is_contiguous() and mask_b.is_contiguous()):
+        raise ValueError("masks must be contiguous CUDA tensors")
+    if scores_a is not None and (scores_a.shape != mask_a.shape or scores_a.dtype != torch.float32 or not scores_a.is_contiguous()):
+        raise ValueError("scores_a must be a contiguous float32 tensor of mask_a's shape")
+    diff = torch.empty_like(mask_a)
+    dsc = torch.empty_like(scores_a) if scores_a is not None else None
+    n = mask_a.numel() // mask_a.shape[-1]
+    stream_mask_difference(n, mask_a.shape[-1], mask_a, scores_a, mask_b.shape[-1], mask_b, diff, dsc, stream)
+    return diff, dsc
+
+
+def effective_k(T: int, block_q: int, s: float) -> int:
+    """Sparsity constant for an effective sparsity ``s`` in [0, 1] (Section 4.2 of the paper):
+    ``k = floor(1 + (T / b_q - 1) s)``, kept inside ``1 .. floor(T / b_q)``. As printed, a larger
+    ``s`` keeps MORE blocks (the prose beside the formula says the opposite; the formula is followed)."""
+    if T < 1 or block_q < 1:
+        raise ValueError("T and block_q must be positive")
+    n = T / block_q
+    return max(1, min(int(1 + (n - 1) * s), max(1, T // block_q)))

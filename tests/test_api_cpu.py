@@ -105,3 +105,10 @@ def test_staging_size_covers_all_buffers(S):
     e = 2
     need = (4 * 256 * 128 * e) * 2 + (2 * 256 * 128 * e) * 2 + 4 * 4 * 4 * 4 + 256
     assert S.stream_host_staging_bytes(p) >= need
+
+
+def test_effective_k_follows_the_printed_formula(S):
+    assert S.effective_k(1000, 32, 0.0) == 1
+    assert S.effective_k(1000, 32, 1.0) == 31          # floor(T / b_q)
+    assert S.effective_k(8192, 32, 0.1) == 26           # floor(1 + 255 * 0.1)
+    assert S.effective_k(64, 64, 0.5) == 1

@@ -303,3 +303,24 @@ def test_vertical_scores_flags_out_of_range_entries(S):
     with pytest.raises(S.StreamError) as e:
         S.vertical_scores(p, mask)
     assert e.value.status == S.STREAM_ERR_DEVICE_CHECK
+
+
+def test_mask_difference_of_two_budgets(S):
+    """Masks built with k = 6 minus masks built with k = 3 on the same inputs, with the larger
+    mask's scores, against the oracle's row-wise difference (integer work: exact)."""
+    w = wl.generate(tc_spec(T=3000, n_q_heads=6, n_kv_heads=2, batch=2, local=True))
+    big = run_mask(S, w, k_top=6, want_scores=True)
+    small = run_mask(S, w, k_top=3)
+    diff, dsc = S.mask_difference(big.mask, small.mask, big.scores)
+    torch.cuda.synchronize()
+    ref, ref_sc = so.mask_difference(big.mask.cpu().numpy().reshape(-1, 6), small.mask.cpu().numpy().reshape(-1, 3),
+                                     big.scores.cpu().numpy().reshape(-1, 6))
+    assert np.array_equal(diff.cpu().numpy().reshape(-1, 6), ref)
+    assert np.array_equal(dsc.cpu().numpy().reshape(-1, 6), ref_sc)
+    assert (ref >= 0).any() and (ref[:, 0] < 0).any()  # both non-trivial and empty rows occur
+    # wide rows, unsorted, with holes: more than one 32-entry sweep on both sides
+    rng = np.random.default_rng(5)
+    a = rng.integers(-1, 300, size=(257, 70)).astype(np.int32)
+    b = rng.integers(-1, 300, size=(257, 45)).astype(np.int32)
+    d2, _ = S.mask_difference(torch.from_numpy(a).cuda(), torch.from_numpy(b).cuda())
+    assert np.array_equal(d2.cpu().numpy(), so.mask_difference(a, b)[0])

@@ -379,3 +379,25 @@ def test_vertical_scores_are_column_sums_with_library_kurtosis():
     # mean 1.75, deviations (2.25, -.75, -.75, -.75): m2 = 1.6875, m4 = 6.64453125 -> 2.3333...
     assert k1[0] == pytest.approx(6.64453125 / 1.6875 ** 2, rel=1e-14)
     assert so.vertical_scores(p1, np.array([[0, -1], [1, -1], [2, -1], [3, -1]], np.int32))[1][0] == 0.0  # flat
+
+
+def test_mask_difference_is_the_row_wise_set_difference():
+    """Pins: numpy's setdiff1d per row (the rows hold distinct blocks), order and scores carried
+    from the first mask, and a hand-worked row."""
+    rng = np.random.default_rng(9)
+    n, ka, kb, nk = 40, 6, 3, 20
+    a = np.stack([rng.permutation(nk)[:ka] for _ in range(n)]).astype(np.int32)
+    b = np.stack([rng.permutation(nk)[:kb] for _ in range(n)]).astype(np.int32)
+    a[rng.random(a.shape) < 0.2] = -1
+    b[rng.random(b.shape) < 0.2] = -1
+    sc = rng.standard_normal(a.shape).astype(np.float32)
+    diff, dsc = so.mask_difference(a, b, sc)
+    for i in range(n):
+        kept = diff[i][diff[i] >= 0]
+        assert sorted(kept.tolist()) == np.setdiff1d(a[i][a[i] >= 0], b[i]).tolist()
+        want = [x for x in a[i].tolist() if x >= 0 and x not in b[i].tolist()]      # order of the first mask
+        assert kept.tolist() == want
+        assert (diff[i][len(kept):] == -1).all() and (dsc[i][len(kept):] == -np.inf).all()
+        assert dsc[i][: len(kept)].tolist() == [float(sc[i][a[i].tolist().index(x)]) for x in want]
+    d, _ = so.mask_difference(np.array([[0, 3, 5, 9, -1, -1]], np.int32), np.array([[0, 9, -1]], np.int32))
+    assert d.tolist() == [[3, 5, -1, -1, -1, -1]]

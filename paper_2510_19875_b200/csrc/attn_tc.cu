@@ -6,25 +6,30 @@
 // rows name one key block each (K_a, K_b, usually different); the tiles arrive by TMA (128-byte
 // swizzle), stacked too, and
 //     S = [Q_0; Q_1] [K_a; K_b]^T      (128 x 128, fp32 in TMEM)
-// holds row 0's logits in its upper-left quadrant and row 1's in its lower-right one. The
-// softmax warps own one TMEM lane (= one query token) per thread pair: they read its 64 logits,
-// apply the element-level mask C, update the running maximum and sum (online softmax, fp32), and
-// write P = exp(.) as bf16 into a block-diagonal 128 x 128 A operand in shared memory whose
-// off-diagonal quadrants stay zero. Then
-//     O_e = P [V_a; V_b]               (128 x 128, fp32 in TMEM, V tiles MN-major)
-// gives both rows' contributions in one chain, which the same threads fold into their fp32
-// output registers (o = o * alpha + O_e) one iteration later, so that the tensor core works on
-// the next logits meanwhile.
+// holds row 0's logits in its upper-left quadrant and row 1's in its lower-right one.
 //
-// Roles (384 threads): warp 0 TMA producer (converged, one elected lane issues); warp 1 issues the Q K^T chains and owns TMEM; warp 3
-// issues the P V chains (two issuing warps, because the thread that issues a chain is held until
-// the tensor core has taken it: with one warp the waits and commits between chains would not
-// overlap with the chains themselves); warp 2 copies the pairs' mask rows from global to shared
-// memory ahead of everyone else; warps 4..11 softmax (two threads per query token: half of its
-// keys and half of its output channels each). Every role walks the same sequence of (pair,
-// entry), read from the shared copy of the mask rows; they meet only on mbarriers. Every wait is
-// bounded: on a timeout the CTA records a code in a device status word, raises a shared abort
-// flag, lets its copies drain and leaves.
+// Two softmax groups of four warps take the entries in turn (entry n belongs to group n % 2), so
+// that one group's chain of waits, TMEM loads, exponentials and fences runs beside the other's.
+// A thread owns one query token (TMEM lane) of its group's entries: it reads the token's 64
+// logits, applies the element-level mask C, and writes P = exp2(scale (s - ref)) as bf16 into
+// its row of the group's 128 x 64 A operand in shared memory. Then two chains with an
+// output-lane mask,
+//     O_g[lanes 0..63]   += P[rows 0..63]   V_a,      O_g[lanes 64..127] += P[rows 64..127] V_b
+// (128 x 128, fp32, accumulated in TMEM per group g; V tiles MN-major), add each row's
+// contribution and leave the other row's lanes alone. `ref` is a per-token reference the group keeps
+// instead of the exact running maximum: it is raised (and the token's O_g lane and sum rescaled
+// in place) only when the maximum has grown by more than a factor 2^8 of exp2's argument, so P
+// stays below 2^8 and rescaling is rare. At the end of a pair the two groups exchange (ref, sum)
+// per token, bring O_0 and O_1 to the common reference, add, normalise and store.
+//
+// Roles (384 threads): warp 0 TMA producer (converged, one elected lane issues; two independent
+// non-blocking load streams, K with Q and V); warp 1 issues the Q K^T chains and owns TMEM; warp 3
+// issues the P V chains (separate issuing warps, because the thread that issues a chain is held
+// until the tensor core has taken it); warp 2 copies the pairs' mask rows from global to shared
+// memory ahead of everyone else; warps 4..7 and 8..11 are the two softmax groups. Every role
+// walks the same sequence of (pair, entry), read from the shared copy of the mask rows; they meet
+// only on mbarriers. Every wait is bounded: on a timeout the CTA records a code in a device
+// status word, raises a shared abort flag, lets its copies drain and leaves.
 #include <math_constants.h>
 
 #include "tc_common.cuh"
@@ -43,28 +48,29 @@ constexpr int kThreads = 384;
 constexpr int kBlk = 64, kD = 128;
 constexpr int kHalfTile = kBlk * 128;       // 64 rows x 128 bytes
 constexpr int kTile = 2 * kHalfTile;        // one 64 x 128 tile
-constexpr int kOperand = 2 * kTile;         // two tiles (K_a, K_b or V_a, V_b), or a 128-row operand
-constexpr int kMaxKStages = 3, kVStages = 2;  // K stages: 3 if shared memory allows, else 2; V stages = O buffers
+constexpr int kOperand = 2 * kTile;         // two tiles (K_a, K_b or V_a, V_b), or the 128-row Q operand
+constexpr int kPBytes = 2 * kHalfTile;      // one group's P: 128 rows x 64 keys
+constexpr int kMaxKStages = 3, kVStages = 2;  // K stages: what shared memory allows (2 or 3); V stages = groups
 constexpr int kMaskSlots = 2;               // pairs whose mask rows are resident
 constexpr int kMaxKTopTc = 1024;
+constexpr float kLazyLog2 = 8.f;            // ref is raised when the maximum exceeds it by this much (log2 units)
 
+// TMEM columns: S of group g at 128 g, O of group g at 256 + 128 g.
 struct Tail {
     unsigned long long q_full, q_empty;
     unsigned long long k_full[kMaxKStages], k_empty[kMaxKStages], v_full[kVStages];
-    // o_full also tells the producer that V stage i is free: the rings of V stages and O buffers
-    // have the same length and move together. There is no "o_empty": P of entry j is published
-    // (p_full) after the same threads folded the product of entry j - 2, and the P V warp waits
-    // for every P before it overwrites that buffer.
-    unsigned long long s_full[2], s_empty[2], o_full[2], p_full;
+    // Per group g (entries n with n % 2 == g): logits ready / read, P published, product added.
+    // o_full[g] also tells the producer that V stage g is free and the group that its P buffer
+    // is: the ring of V stages and the groups move together.
+    unsigned long long s_full[2], s_empty[2], p_full[2], o_full[2];
     unsigned long long m_full[kMaskSlots], m_empty[kMaskSlots];
-    unsigned long long x_bar[4];  // softmax warps w and w + 4 meet here
+    unsigned long long x_bar[4];  // the two softmax warps of a lane quarter (one per group) meet here
     unsigned int tmem_base;
     int abort_flag;
-    float xch[2][128][2];         // their exchange slots: [buffer][token][part]
 };
-// Dynamic shared memory: Q | P | V stages | K stages | Tail | mask rows [kMaskSlots][2][row_stride]
-// (-1 where a row has nothing), the first four 1024-byte aligned.
-constexpr int kFixedOperands = 2 + kVStages;
+// Dynamic shared memory: Q | P of group 0, P of group 1 | V stages | K stages | Tail | mask rows
+// [kMaskSlots][2][row_stride] (-1 where a row has nothing), the operands 1024-byte aligned.
+constexpr int kFixedOperands = 2 + kVStages;  // Q, the two P together, the V stages
 constexpr int kMaxSmemPerCta = 232448;
 
 constexpr unsigned kIdescQK = idesc_bf16(128, 128, false);  // B = stacked K tiles, K-major
@@ -272,7 +278,7 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
 // The two issuing roles are run by all 32 lanes of their warps, converged: the waits are
 // warp-wide, one elected lane issues.
 
-// S = [Q_0; Q_1] [K_a; K_b]^T for every kept entry.
+// S_g = [Q_0; Q_1] [K_a; K_b]^T for every kept entry (g = entry count % 2, over the whole kernel).
 __device__ void qk_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_smem, unsigned tmem_base) {
     const Geom &g = P.g;
     Ring ks, sb, ms;
@@ -315,11 +321,10 @@ __device__ void qk_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_s
     }
 }
 
-// O = P [V_a; V_b] for every kept entry.
+// O_g (+)= P_g [V_a; V_b] for every kept entry; a group's first entry of a pair starts its O afresh.
 __device__ void pv_role(const Params &P, Tail *tl, unsigned p_smem, unsigned v_smem, unsigned tmem_base) {
     const Geom &g = P.g;
-    Ring vs, ob, ms;
-    unsigned p_par = 0;
+    Ring gr, ms;  // gr: group = V stage = O buffer of the entry
     // the MN-major V tiles have their two 64-channel halves kHalfTile apart
     const unsigned p_lo = desc_lo_sw128(p_smem, 16), v_lo = desc_lo_sw128(v_smem, kHalfTile);
     for (int id = blockIdx.x; id < P.n_items; id += gridDim.x) {
@@ -327,24 +332,29 @@ __device__ void pv_role(const Params &P, Tail *tl, unsigned p_smem, unsigned v_s
         const int *rows = mask_rows(tl, P, ms.idx);
         Entry cur;
         int e = next_entry(rows, P.row_stride, -1, g.k_top, &cur);
+        unsigned fresh = 3u;  // bit g: group g has not added anything for this pair yet
         while (e < g.k_top) {
             e = next_entry(rows, P.row_stride, e, g.k_top, &cur);
-            if (!wait_w(smem_u32(&tl->v_full[vs.idx]), vs.phase, tl, 205)) return;
-            if (!wait_w(smem_u32(&tl->p_full), p_par, tl, 204)) return;  // also: O buffer ob has been folded
-            p_par ^= 1;
+            if (!wait_w(smem_u32(&tl->v_full[gr.idx]), gr.phase, tl, 205)) return;
+            if (!wait_w(smem_u32(&tl->p_full[gr.idx]), gr.phase, tl, 204)) return;  // also: O_g rescaled if it had to be
             tc_fence_after();
-            const unsigned d_tmem = tmem_base + 256 + ob.idx * 128;
-            const unsigned b_lo = v_lo + vs.idx * (kOperand >> 4);
+            const unsigned d_tmem = tmem_base + 256 + gr.idx * 128;
+            const unsigned a_lo = p_lo + gr.idx * (kPBytes >> 4), b_lo = v_lo + gr.idx * (kOperand >> 4);
+            const unsigned keep = ((fresh >> gr.idx) & 1u) ^ 1u;
+            fresh &= ~(1u << gr.idx);
             if (elect_one()) {
 #pragma unroll
-                for (int s = 0; s < 8; ++s)  // 16 keys per step: P column half = V tile = s / 4
-                    tc_mma_bf16_split(d_tmem, p_lo + (((s >> 2) * 2 * kHalfTile + (s & 3) * 32) >> 4), kHiK,
-                                      b_lo + (((s >> 2) * kTile + (s & 3) * 2048) >> 4), kHiK, kIdescPV, s != 0);
-                tc_commit(smem_u32(&tl->o_full[ob.idx]));  // product ready = V stage and P buffer free
+                for (int tile = 0; tile < 2; ++tile) {  // row `tile` of the pair: its P rows, its V tile, its lanes
+                    const unsigned lo_off = tile ? 0xFFFFFFFFu : 0u, hi_off = tile ? 0u : 0xFFFFFFFFu;
+#pragma unroll
+                    for (int s4 = 0; s4 < 4; ++s4)  // 16 keys per step
+                        tc_mma_bf16_split_masked(d_tmem, a_lo + ((s4 * 32) >> 4), kHiK, b_lo + ((tile * kTile + s4 * 2048) >> 4),
+                                                 kHiK, kIdescPV, s4 != 0 ? 1u : keep, lo_off, lo_off, hi_off, hi_off);
+                }
+                tc_commit(smem_u32(&tl->o_full[gr.idx]));  // product added = V stage and P buffer of the group free
             }
             __syncwarp();
-            ob.advance(2);
-            vs.advance(kVStages);
+            gr.advance(2);
         }
         if (elect_one()) mbar_arrive(smem_u32(&tl->m_empty[ms.idx]));
         __syncwarp();
@@ -365,70 +375,65 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
     return y;
 }
 
-// o[0..63] = o * alpha + O, O being 64 columns of this thread's lane of a TMEM buffer.
-__device__ __forceinline__ void fold_output(float *o, float alpha, unsigned taddr) {
-    unsigned r[64];
-    tmem_ld_32x32_issue(taddr, r);
-    tmem_ld_32x32_issue(taddr + 32, r + 32);
-    tmem_ld_wait();
+// Multiplies 128 fp32 columns of this thread's TMEM lane by f, in place (every lane of the warp
+// takes part; lanes that need no change pass f = 1).
+__device__ __forceinline__ void rescale_lane(unsigned taddr, float f) {
+#pragma unroll 1
+    for (int c = 0; c < 4; ++c) {
+        unsigned r[32];
+        tmem_ld_32x32_issue(taddr + c * 32, r);
+        tmem_ld_wait();
 #pragma unroll
-    for (int i = 0; i < 64; ++i) o[i] = fmaf(o[i], alpha, __uint_as_float(r[i]));
+        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * f);
+        tmem_st_32x32_issue(taddr + c * 32, r);
+    }
+    tmem_st_wait();
 }
 
-// Eight softmax warps. Warps w and w + 4 share the 32 TMEM lanes (query tokens) 32 (w % 4) ..: the
-// first takes keys 0..31 of the token's block and output channels 0..63, the second keys 32..63
-// and channels 64..127. Both read all 64 logits for the row maximum, so they only have to meet
-// once per pair, to add up their partial sums (through shared memory, on an mbarrier of their own).
+// One softmax group: four warps, thread = query token (TMEM lane) `row` of the pair, for the
+// entries n with n % 2 == grp (n counts the kept entries over the whole kernel, as in every role).
+// The waits are warp-wide (same answer in every lane), so the warp stays converged for the
+// warp-collective TMEM loads and stores and leaves together if the CTA aborts.
 __device__ void softmax_role(const Params &P, Tail *tl, unsigned char *p_ptr, unsigned tmem_base, int t) {
     const Geom &g = P.g;
-    const int lane = t & 31, row = t & 127, part = t >> 7, half = row >> 6, mq = row & 63, wq = row >> 5;
+    const int lane = t & 31, row = t & 127, grp = t >> 7, half = row >> 6, mq = row & 63, wq = row >> 5;
     const unsigned lane_off = (unsigned)(row & ~31) << 16;
-    // this thread's row of the block-diagonal P operand: column half = its row of the pair
-    unsigned char *p_row = p_ptr + half * 2 * kHalfTile + (row >> 3) * 1024 + (row & 7) * 128;
+    // this thread's row of its group's P operand, and the same row in the other group's: the two
+    // exchange a few bytes there at the end of a pair
+    const int row_off = (row >> 3) * 1024 + (row & 7) * 128;
+    unsigned char *p_row = p_ptr + grp * kPBytes + row_off;
+    const unsigned char *p_row_other = p_ptr + (grp ^ 1) * kPBytes + row_off;
     const int sw = row & 7;
-    const unsigned x_bar = smem_u32(&tl->x_bar[wq]);
-    unsigned x_par = 0;
-    int x_buf = 0;
-    // publish v, meet the partner warp, return the partner's value
-    auto exchange = [&](float v, float *other) -> bool {
-        tl->xch[x_buf][row][part] = v;
-        __syncwarp();
-        if (lane == 0) mbar_arrive(x_bar);
-        if (!wait(x_bar, x_par, tl, 304)) return false;
-        x_par ^= 1;
-        *other = tl->xch[x_buf][row][part ^ 1];
-        x_buf ^= 1;
-        return true;
-    };
-    Ring sb, ob, ms;
+    const unsigned s_full = smem_u32(&tl->s_full[grp]), s_empty = smem_u32(&tl->s_empty[grp]),
+                   p_full = smem_u32(&tl->p_full[grp]), o_full = smem_u32(&tl->o_full[grp]), x_bar = smem_u32(&tl->x_bar[wq]);
+    const unsigned s_addr = tmem_base + grp * 128 + half * 64 + lane_off;
+    const unsigned o_own = tmem_base + 256 + grp * 128 + lane_off, o_other = tmem_base + 256 + (grp ^ 1) * 128 + lane_off;
+    unsigned s_par = 0, o_par = 0, x_par = 0;
+    unsigned n = 0;  // kept entries so far
+    Ring ms;
     for (int id = blockIdx.x; id < P.n_items; id += gridDim.x) {
         const Item it = decode_item(P, id);
         const long long tq = (long long)it.qb * kBlk + mq;
         const bool row_active = half < it.R && tq < g.T;
-        if (!wait(smem_u32(&tl->m_full[ms.idx]), ms.phase, tl, 305)) return;
+        if (!wait_w(smem_u32(&tl->m_full[ms.idx]), ms.phase, tl, 305)) return;
         const int *rows = mask_rows(tl, P, ms.idx);
-        float o[64];
-#pragma unroll
-        for (int i = 0; i < 64; ++i) o[i] = 0.f;
-        float m = -CUDART_INF_F, l = 0.f, alpha_prev = 1.f;
-        bool have_prev = false;
-        Entry cur, nxt;
-        int e = next_entry(rows, P.row_stride, -1, g.k_top, &cur);
-        while (e < g.k_top) {
-            const int e_next = next_entry(rows, P.row_stride, e, g.k_top, &nxt);  // its latency hides behind the wait
-            // this token's 64 logits against its row's key block: both threads of the token read
-            // all of them for the row maximum; each then exponentiates its own 32
-            if (!wait(smem_u32(&tl->s_full[sb.idx]), sb.phase, tl, 301)) return;
+        float ref = -CUDART_INF_F, l = 0.f;
+        bool pending = false;  // a P V chain of this group and pair may still be running
+        Entry cur;
+        for (int e = next_entry(rows, P.row_stride, -1, g.k_top, &cur); e < g.k_top;
+             e = next_entry(rows, P.row_stride, e, g.k_top, &cur), ++n) {
+            if ((int)(n & 1u) != grp) continue;
+            // the token's 64 logits against its row's key block
+            if (!wait_w(s_full, s_par, tl, 301)) return;
+            s_par ^= 1;
             tc_fence_after();
             unsigned sr[64];
-            const unsigned s_addr = tmem_base + sb.idx * 128 + half * 64 + lane_off;
-            tmem_ld_32x32_issue(s_addr + part * 32, sr);             // own keys first
-            tmem_ld_32x32_issue(s_addr + (part ^ 1) * 32, sr + 32);  // the partner's
+            tmem_ld_32x32_issue(s_addr, sr);
+            tmem_ld_32x32_issue(s_addr + 32, sr + 32);
             tmem_ld_wait();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&tl->s_empty[sb.idx]));
-            sb.advance(2);
+            if (lane == 0) mbar_arrive(s_empty);
             // keys of the block this token may attend: a prefix of n_hi keys (inside T, not after it if causal)
             const int blk = half ? cur.b : cur.a;
             int n_hi = 0;
@@ -438,7 +443,6 @@ __device__ void softmax_role(const Params &P, Tail *tl, unsigned char *p_ptr, un
                 if (g.causal) lim = min(lim, tq - k0 + 1);
                 n_hi = (int)max(0ll, min(lim, (long long)kBlk));
             }
-            const int n_own = n_hi - part * 32, n_oth = n_hi - (part ^ 1) * 32;  // within each half
             const bool all_keys = n_hi == kBlk;  // every block but the diagonal one and the one across T
             float mx4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
             if (all_keys) {
@@ -451,20 +455,32 @@ __device__ void softmax_role(const Params &P, Tail *tl, unsigned char *p_ptr, un
                 }
             } else {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    mx4[i & 3] = fmaxf(mx4[i & 3], i < n_own ? __uint_as_float(sr[i]) : -CUDART_INF_F);
-                    mx4[i & 3] = fmaxf(mx4[i & 3], i < n_oth ? __uint_as_float(sr[32 + i]) : -CUDART_INF_F);
-                }
+                for (int i = 0; i < 64; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], i < n_hi ? __uint_as_float(sr[i]) : -CUDART_INF_F);
             }
-            const float m_new = fmaxf(m, fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])));
-            // with no key allowed so far m_new is -inf: every p is 0 and nothing is rescaled
-            const float shift = m_new == -CUDART_INF_F ? 0.f : -m_new * P.scale_log2;
-            const float alpha = m_new == m ? 1.f : fast_exp2((m - m_new) * P.scale_log2);
+            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+            // the reference: the first allowed logits set it; later it only moves when the maximum
+            // has outgrown it by kLazyLog2, and then what the group has accumulated is rescaled
+            const bool raise = ref != -CUDART_INF_F && (mx - ref) * P.scale_log2 > kLazyLog2;
+            const float new_ref = (ref == -CUDART_INF_F || raise) ? mx : ref;
+            // this group's previous chain of the pair must be done before its P buffer is rewritten
+            // or its O lane rescaled
+            if (pending) {
+                if (!wait_w(o_full, o_par, tl, 302)) return;
+                o_par ^= 1;
+                tc_fence_after();
+            }
+            if (__any_sync(0xffffffffu, raise)) {
+                const float f = raise ? fast_exp2((ref - new_ref) * P.scale_log2) : 1.f;
+                rescale_lane(o_own, f);
+                l *= f;
+            }
+            ref = new_ref;
+            const float shift = ref == -CUDART_INF_F ? 0.f : -ref * P.scale_log2;
             float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-            unsigned packed[16];
+            unsigned packed[32];
             if (all_keys) {
 #pragma unroll
-                for (int i = 0; i < 32; i += 2) {
+                for (int i = 0; i < 64; i += 2) {
                     const float p0 = fast_exp2(fmaf(__uint_as_float(sr[i]), P.scale_log2, shift));
                     const float p1 = fast_exp2(fmaf(__uint_as_float(sr[i + 1]), P.scale_log2, shift));
                     sum4[(i >> 1) & 3] += p0 + p1;
@@ -473,65 +489,84 @@ __device__ void softmax_role(const Params &P, Tail *tl, unsigned char *p_ptr, un
                 }
             } else {
 #pragma unroll
-                for (int i = 0; i < 32; i += 2) {
+                for (int i = 0; i < 64; i += 2) {
                     float p0 = fast_exp2(fmaf(__uint_as_float(sr[i]), P.scale_log2, shift));
                     float p1 = fast_exp2(fmaf(__uint_as_float(sr[i + 1]), P.scale_log2, shift));
-                    p0 = i < n_own ? p0 : 0.f;
-                    p1 = i + 1 < n_own ? p1 : 0.f;
+                    p0 = i < n_hi ? p0 : 0.f;
+                    p1 = i + 1 < n_hi ? p1 : 0.f;
                     sum4[(i >> 1) & 3] += p0 + p1;
                     __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
                     packed[i >> 1] = *reinterpret_cast<unsigned *>(&pk);
                 }
             }
-            l = l * alpha + ((sum4[0] + sum4[1]) + (sum4[2] + sum4[3]));
-            m = m_new;
-            // the P buffer is free, and the previous product ready, once the previous P V chain is done
-            if (have_prev) {
-                if (!wait(smem_u32(&tl->o_full[ob.idx]), ob.phase, tl, 302)) return;
-                tc_fence_after();
-            }
+            l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
-                *reinterpret_cast<uint4 *>(p_row + (((part * 4 + c) ^ sw) << 4)) =
+            for (int c = 0; c < 8; ++c)
+                *reinterpret_cast<uint4 *>(p_row + ((c ^ sw) << 4)) =
                     make_uint4(packed[4 * c], packed[4 * c + 1], packed[4 * c + 2], packed[4 * c + 3]);
             fence_async_smem();
-            tc_fence_before();  // this thread's TMEM reads (the product folded last round) are done
+            tc_fence_before();  // the rescaled O lane, if any, is in place
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&tl->p_full));
-            if (have_prev) {
-                fold_output(o, alpha_prev, tmem_base + 256 + ob.idx * 128 + part * 64 + lane_off);
-                ob.advance(2);
-            }
-            alpha_prev = alpha;
-            have_prev = true;
-            e = e_next;
-            cur = nxt;
+            if (lane == 0) mbar_arrive(p_full);
+            pending = true;
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&tl->m_empty[ms.idx]));
         ms.advance(kMaskSlots);
-        if (have_prev) {
-            if (!wait(smem_u32(&tl->o_full[ob.idx]), ob.phase, tl, 303)) return;
+        // End of the pair: bring the two groups' sums to a common reference and store.
+        if (pending) {
+            if (!wait_w(o_full, o_par, tl, 303)) return;
+            o_par ^= 1;
             tc_fence_after();
-            fold_output(o, alpha_prev, tmem_base + 256 + ob.idx * 128 + part * 64 + lane_off);
-            ob.advance(2);
         }
-        float l_other;
-        if (!exchange(l, &l_other)) return;
-        if (row_active) {
-            const float lt = l + l_other;
-            const float inv = lt > 0.f ? 1.f / lt : 0.f;
-            uint4 *dst = reinterpret_cast<uint4 *>(P.out + (((long long)it.b * g.H + it.h0 + half) * g.T + tq) * kD + part * 64);
+        *reinterpret_cast<float2 *>(p_row) = make_float2(ref, l);  // the P row is free: use it as mailbox
+        __syncwarp();
+        if (lane == 0) mbar_arrive(x_bar);
+        if (!wait_w(x_bar, x_par, tl, 304)) return;
+        x_par ^= 1;
+        tc_fence_after();  // the other group's last chain is complete too
+        const float2 oth = *reinterpret_cast<const float2 *>(p_row_other);
+        const float top = fmaxf(ref, oth.x);
+        const float f_own = ref == -CUDART_INF_F ? 0.f : fast_exp2((ref - top) * P.scale_log2);
+        const float f_oth = oth.x == -CUDART_INF_F ? 0.f : fast_exp2((oth.x - top) * P.scale_log2);
+        const float total = l * f_own + oth.y * f_oth;
+        const float inv = total > 0.f ? 1.f / total : 0.f;
+        const float w_own = f_own * inv, w_oth = f_oth * inv;
+        // this group stores channels 64 grp .. 64 grp + 63 of every token
+        uint4 out_words[8];
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {
+        for (int c = 0; c < 2; ++c) {
+            unsigned ra[32], rb[32];
+            tmem_ld_32x32_issue(o_own + grp * 64 + c * 32, ra);
+            tmem_ld_32x32_issue(o_other + grp * 64 + c * 32, rb);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
                 unsigned w[4];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    __nv_bfloat162 pk = __floats2bfloat162_rn(o[8 * c + 2 * j] * inv, o[8 * c + 2 * j + 1] * inv);
-                    w[j] = *reinterpret_cast<unsigned *>(&pk);
+                for (int u = 0; u < 4; ++u) {
+                    const int i = 8 * j + 2 * u;
+                    // a group without entries in this pair holds stale numbers: weight 0 means "leave out"
+                    const float a0 = w_own != 0.f ? __uint_as_float(ra[i]) * w_own : 0.f;
+                    const float a1 = w_own != 0.f ? __uint_as_float(ra[i + 1]) * w_own : 0.f;
+                    const float v0 = w_oth != 0.f ? fmaf(__uint_as_float(rb[i]), w_oth, a0) : a0;
+                    const float v1 = w_oth != 0.f ? fmaf(__uint_as_float(rb[i + 1]), w_oth, a1) : a1;
+                    __nv_bfloat162 pk = __floats2bfloat162_rn(v0, v1);
+                    w[u] = *reinterpret_cast<unsigned *>(&pk);
                 }
-                dst[c] = make_uint4(w[0], w[1], w[2], w[3]);
+                out_words[c * 4 + j] = make_uint4(w[0], w[1], w[2], w[3]);
             }
+        }
+        // second meeting: both groups have read both O buffers and both mailboxes
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(x_bar);
+        if (!wait_w(x_bar, x_par, tl, 306)) return;
+        x_par ^= 1;
+        if (row_active) {
+            uint4 *dst = reinterpret_cast<uint4 *>(P.out + (((long long)it.b * g.H + it.h0 + half) * g.T + tq) * kD + grp * 64);
+#pragma unroll
+            for (int c = 0; c < 8; ++c) dst[c] = out_words[c];
         }
     }
 }
@@ -544,7 +579,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     // what is left behind the aligned base decides the number of K stages (the same in every thread)
     const int fixed_bytes = (int)(smem - smem_raw) + (int)sizeof(Tail) + kMaskSlots * 2 * P.row_stride * (int)sizeof(int);
     P.n_k_stages = min(kMaxKStages, (P.smem_bytes - fixed_bytes) / kOperand - kFixedOperands);
-    const unsigned q_smem = smem_u32(smem), p_smem = q_smem + kOperand, v_smem = p_smem + kOperand,
+    const unsigned q_smem = smem_u32(smem), p_smem = q_smem + kOperand, v_smem = p_smem + 2 * kPBytes,
                    k_smem = v_smem + kVStages * kOperand;
     Tail *tl = (Tail *)(smem + (kFixedOperands + P.n_k_stages) * kOperand);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -555,19 +590,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         for (int i = 0; i < kMaxKStages; ++i) { mbar_init(smem_u32(&tl->k_full[i]), 1); mbar_init(smem_u32(&tl->k_empty[i]), 1); }
         for (int i = 0; i < kVStages; ++i) mbar_init(smem_u32(&tl->v_full[i]), 1);
         for (int i = 0; i < 2; ++i) {
-            mbar_init(smem_u32(&tl->s_full[i]), 1); mbar_init(smem_u32(&tl->s_empty[i]), 8);
-            mbar_init(smem_u32(&tl->o_full[i]), 1);
+            mbar_init(smem_u32(&tl->s_full[i]), 1); mbar_init(smem_u32(&tl->s_empty[i]), 4);
+            mbar_init(smem_u32(&tl->p_full[i]), 4); mbar_init(smem_u32(&tl->o_full[i]), 1);
         }
-        mbar_init(smem_u32(&tl->p_full), 8);
         for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&tl->x_bar[i]), 2);
         for (int i = 0; i < kMaskSlots; ++i) { mbar_init(smem_u32(&tl->m_full[i]), 1); mbar_init(smem_u32(&tl->m_empty[i]), 12); }
         tl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    // P starts as zeros: its off-diagonal quadrants are never written again
-    for (int i = threadIdx.x; i < kOperand / 16; i += kThreads)
-        reinterpret_cast<uint4 *>(smem + kOperand)[i] = make_uint4(0, 0, 0, 0);
-    fence_async_smem();
     if (warp == 1) tmem_alloc_512(smem_u32(&tl->tmem_base));  // all columns: one CTA per SM
     tc_fence_before();
     __syncthreads();

@@ -137,6 +137,19 @@ __device__ __forceinline__ void tc_mma_bf16_split(unsigned d_tmem, unsigned a_lo
         : "memory");
 }
 
+// The same with an output-lane mask: bit i of the 128-bit vector {m0 (lanes 0..31), m1, m2, m3}
+// set = accumulator lane i is left untouched by this instruction.
+__device__ __forceinline__ void tc_mma_bf16_split_masked(unsigned d_tmem, unsigned a_lo, unsigned a_hi, unsigned b_lo,
+                                                         unsigned b_hi, unsigned idesc, unsigned accumulate, unsigned m0,
+                                                         unsigned m1, unsigned m2, unsigned m3) {
+    asm volatile(
+        "{\n.reg .pred p;\n.reg .b64 da, db;\nmov.b64 da, {%1, %2};\nmov.b64 db, {%3, %4};\nsetp.ne.b32 p, %6, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, {%7, %8, %9, %10}, p;\n}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate), "r"(m0), "r"(m1), "r"(m2),
+          "r"(m3)
+        : "memory");
+}
+
 __device__ __forceinline__ void tmem_alloc_512(unsigned smem_dst) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(512) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -169,6 +182,20 @@ __device__ __forceinline__ void tmem_ld_32x16_issue(unsigned taddr, unsigned *r)
         : "r"(taddr)
         : "memory");
 }
+// Store 32 consecutive fp32 columns of this thread's TMEM lane (the inverse of the load above).
+// Complete for later tcgen05 operations after tmem_st_wait().
+__device__ __forceinline__ void tmem_st_32x32_issue(unsigned taddr, const unsigned *r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
+          "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
+          "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 __device__ __forceinline__ void tmem_ld_32x32(unsigned taddr, float *v) {

@@ -137,6 +137,18 @@ __device__ __forceinline__ int next_entry(const int *rows, int stride, int e, in
     return k_top;
 }
 
+// Number of kept entries of a pair, counted by a converged warp (32 entries per ballot).
+__device__ __forceinline__ int count_entries(const int *rows, int stride, int k_top) {
+    const int lane = threadIdx.x & 31;
+    int n = 0;
+    for (int base = 0; base < k_top; base += 32) {
+        const int e = base + lane;
+        const bool kept = e < k_top && (rows[e] >= 0 || rows[stride + e] >= 0);
+        n += __popc(__ballot_sync(0xffffffffu, kept));
+    }
+    return n;
+}
+
 // ----------------------------------------------------------------------------------------------
 // Roles. All walk the kept entries x_0 .. x_{n-1} of a pair in "rounds": round r handles the
 // logits of x_r and the P V product of x_{r-1}.
@@ -287,14 +299,12 @@ __device__ void qk_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_s
     for (int id = blockIdx.x; id < P.n_items; id += gridDim.x) {
         if (!wait_w(smem_u32(&tl->m_full[ms.idx]), ms.phase, tl, 207)) return;
         const int *rows = mask_rows(tl, P, ms.idx);
-        Entry cur;
-        int e = next_entry(rows, P.row_stride, -1, g.k_top, &cur);
-        if (e < g.k_top) {
+        const int n_entries = count_entries(rows, P.row_stride, g.k_top);  // the issuers need no more than the count
+        if (n_entries > 0) {
             if (!wait_w(smem_u32(&tl->q_full), q_par, tl, 201)) return;
             q_par ^= 1;
         }
-        while (e < g.k_top) {
-            e = next_entry(rows, P.row_stride, e, g.k_top, &cur);  // (only "is there another entry" matters here)
+        for (int i = 0; i < n_entries; ++i) {
             if (!wait_w(smem_u32(&tl->k_full[ks.idx]), ks.phase, tl, 202)) return;
             if (!wait_w(smem_u32(&tl->s_empty[sb.idx]), sb.phase ^ 1, tl, 203)) return;
             tc_fence_after();
@@ -309,7 +319,7 @@ __device__ void qk_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_s
                                           b_lo + ((c * 2 * kHalfTile + k4 * 32) >> 4), kHiK, kIdescQK, (c | k4) != 0);
                 tc_commit(smem_u32(&tl->s_full[sb.idx]));
                 tc_commit(smem_u32(&tl->k_empty[ks.idx]));
-                if (e >= g.k_top) tc_commit(smem_u32(&tl->q_empty));  // that was the pair's last use of Q
+                if (i + 1 == n_entries) tc_commit(smem_u32(&tl->q_empty));  // that was the pair's last use of Q
             }
             __syncwarp();
             sb.advance(2);
@@ -330,11 +340,9 @@ __device__ void pv_role(const Params &P, Tail *tl, unsigned p_smem, unsigned v_s
     for (int id = blockIdx.x; id < P.n_items; id += gridDim.x) {
         if (!wait_w(smem_u32(&tl->m_full[ms.idx]), ms.phase, tl, 208)) return;
         const int *rows = mask_rows(tl, P, ms.idx);
-        Entry cur;
-        int e = next_entry(rows, P.row_stride, -1, g.k_top, &cur);
+        const int n_entries = count_entries(rows, P.row_stride, g.k_top);
         unsigned fresh = 3u;  // bit g: group g has not added anything for this pair yet
-        while (e < g.k_top) {
-            e = next_entry(rows, P.row_stride, e, g.k_top, &cur);
+        for (int i = 0; i < n_entries; ++i) {
             if (!wait_w(smem_u32(&tl->v_full[gr.idx]), gr.phase, tl, 205)) return;
             if (!wait_w(smem_u32(&tl->p_full[gr.idx]), gr.phase, tl, 204)) return;  // also: O_g rescaled if it had to be
             tc_fence_after();

@@ -35,10 +35,21 @@ constexpr int kHalfTile = kBlk * 128;          // 64 rows x 128 bytes (one 64-ch
 constexpr int kStageBytes = 4 * kHalfTile;     // [2 channel halves][2 tiles]
 constexpr int kQBytes = 2 * kR * kHalfTile;    // [2 channel halves][kR rows]
 constexpr int kMaxJobs = 64;
+constexpr int kListReaders = 1 + kMmaWarps + 4;  // producer warp, MMA warps, epilogue warps
+// A parity wait only means something to a thread that saw the phase before it complete. Chain c
+// goes to warp c % kMmaWarps and slot c % kSlots, so with this a warp is the only issuer that
+// ever waits on its slots and meets every phase of them.
+static_assert(kSlots % kMmaWarps == 0, "each TMEM slot must always meet the same issuing warp");
 
 struct Tail {
     unsigned long long full[kStages], empty[kStages], tmem_full[kSlots], tmem_empty[kSlots];
     unsigned long long q_full, jobs_ready[kR + 1], scores_done[kR];
+    // jobs_ack[i]: every reader of list i (the producer, the MMA warps, the epilogue warps) has
+    // taken what it needs from n_jobs[i], jobs_blk[i] and, for i = kR, the group record; the
+    // controller waits for it before it writes them again. Without it a warp with nothing to do
+    // in a short list could still be about to read it when the next one is written, or fall two
+    // phases behind jobs_ready[i].
+    unsigned long long jobs_ack[kR + 1];
     unsigned int tmem_base;
     int abort_flag;
     int grp_id, grp_b, grp_kvh, grp_qb, grp_h0, grp_R;
@@ -123,6 +134,8 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
                     __syncwarp();
                     st.advance(kStages);
                 }
+                if (elect_one()) mbar_arrive(smem_u32(&tl->jobs_ack[li]));  // done reading this list
+                __syncwarp();
             }
         }
     }
@@ -155,16 +168,21 @@ __device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_
                     jr_par[x] ^= 1;
                 }
                 const int n = tl->n_jobs[li];
+                __syncwarp();
+                if (elect_one()) mbar_arrive(smem_u32(&tl->jobs_ack[li]));  // the count is all this role reads
+                __syncwarp();
                 for (int j = 0; j < n; j += 2) {
                     const int r0 = level == 0 ? 0 : x, r1 = level == 0 ? R : x + 1;
-                    bool stage_ready = false;
+                    // Every issuing warp waits for every stage, with or without a chain in it: it
+                    // then sees each phase of full[] in turn (a warp that skipped some could take a
+                    // phase still in flight for the one after it), and its arrival on empty[] cannot
+                    // come before the stage's previous use was released.
+                    if (!mbar_wait_w(smem_u32(&tl->full[st.idx]), st.phase, tl, P.ws, 204)) return;
+                    bool issued = false;
                     const unsigned a_lo = desc_lo_sw128(k_smem + st.idx * kStageBytes, 16);
                     for (int r = r0; r < r1; ++r, ++chain, sl.advance(kSlots)) {
                         if ((int)(chain % kMmaWarps) != which) continue;
-                        if (!stage_ready) {
-                            if (!mbar_wait_w(smem_u32(&tl->full[st.idx]), st.phase, tl, P.ws, 204)) return;
-                            stage_ready = true;
-                        }
+                        issued = true;
                         if (!mbar_wait_w(smem_u32(&tl->tmem_empty[sl.idx]), sl.phase ^ 1, tl, P.ws, 205)) return;
                         tc_fence_after();
                         const unsigned d_tmem = tmem_base + sl.idx * 64;
@@ -183,7 +201,7 @@ __device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_
                     // the stage is free once every issuing warp is done with it: those that read it
                     // commit behind their chains, the others just arrive
                     if (elect_one()) {
-                        if (stage_ready) tc_commit(smem_u32(&tl->empty[st.idx]));
+                        if (issued) tc_commit(smem_u32(&tl->empty[st.idx]));
                         else mbar_arrive(smem_u32(&tl->empty[st.idx]));
                     }
                     __syncwarp();
@@ -254,6 +272,7 @@ __device__ void epilogue_role(const Params &P, Tail *tl, unsigned tmem_base, int
                 if (lane == 0) {
                     const int r0 = level == 0 ? 0 : x, r1 = level == 0 ? R : x + 1;
                     for (int r = r0; r < r1; ++r) mbar_arrive(smem_u32(&tl->scores_done[r]));
+                    mbar_arrive(smem_u32(&tl->jobs_ack[li]));  // done reading this list
                 }
             }
         }
@@ -284,6 +303,7 @@ __device__ void controller_role(const Params &P, Tail *tl, int lane) {
     const Geom &g = P.g;
     const unsigned lt = (1u << lane) - 1u;
     unsigned sd_par[kR] = {0, 0, 0, 0};
+    unsigned ack_par[kR + 1] = {0, 0, 0, 0, 0};  // phase of the next acknowledgement of each list
     for (;;) {
         int id = 0;
         if (lane == 0) id = (int)atomicAdd(&P.ws->work_counter, 1u);
@@ -307,6 +327,9 @@ __device__ void controller_role(const Params &P, Tail *tl, int lane) {
         const bool vl1 = v0, vr1 = v0 && m0 + 1 <= l0 && m0 + 1 <= q_lim;
         const unsigned bl = __ballot_sync(0xffffffffu, vl1), br = __ballot_sync(0xffffffffu, vr1);
         const int c_l1 = __popc(bl & lt) + __popc(br & lt), c_r1 = c_l1 + (vl1 ? 1 : 0);
+        // the previous group's first list and record have been read by everybody (passes at once the first time)
+        if (!mbar_wait(smem_u32(&tl->jobs_ack[kR]), ack_par[kR] ^ 1, tl, P.ws, 402)) return;
+        ack_par[kR] ^= 1;
         if (vl1) tl->jobs_blk[kR][c_l1] = f0;
         if (vr1) tl->jobs_blk[kR][c_r1] = m0 + 1;
         const int n1 = __popc(bl) + __popc(br);
@@ -360,6 +383,8 @@ __device__ void controller_role(const Params &P, Tail *tl, int lane) {
                     has_r[r] = live && nl[r] > nf[r] && mm + 1 <= q_lim;
                     const unsigned hb = __ballot_sync(0xffffffffu, has_r[r]);
                     my_c[r] = __popc(hb & lt);
+                    if (!mbar_wait(smem_u32(&tl->jobs_ack[r]), ack_par[r] ^ 1, tl, P.ws, 403)) return;
+                    ack_par[r] ^= 1;
                     if (has_r[r]) tl->jobs_blk[r][my_c[r]] = mm + 1;
                     if (lane == 0) tl->n_jobs[r] = __popc(hb);
                     tiles += (unsigned)__popc(hb);
@@ -394,7 +419,7 @@ mask_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         for (int i = 0; i < kStages; ++i) { mbar_init(smem_u32(&tl->full[i]), 1); mbar_init(smem_u32(&tl->empty[i]), kMmaWarps); }
         for (int i = 0; i < kSlots; ++i) { mbar_init(smem_u32(&tl->tmem_full[i]), 1); mbar_init(smem_u32(&tl->tmem_empty[i]), 4); }
         mbar_init(smem_u32(&tl->q_full), 1);
-        for (int i = 0; i <= kR; ++i) mbar_init(smem_u32(&tl->jobs_ready[i]), 1);
+        for (int i = 0; i <= kR; ++i) { mbar_init(smem_u32(&tl->jobs_ready[i]), 1); mbar_init(smem_u32(&tl->jobs_ack[i]), kListReaders); }
         for (int i = 0; i < kR; ++i) mbar_init(smem_u32(&tl->scores_done[i]), 4);
         tl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");

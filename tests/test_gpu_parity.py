@@ -35,6 +35,8 @@ def assert_mask_parity(S, w, rows, *, impl="auto", score_cache=True, **kw):
     spec = w.spec
     res = run_mask(S, w, impl=impl, want_scores=True, **kw)
     mask = res.mask.cpu().numpy()
+    st = res.stats()
+    assert st.error == 0, f"device error {st.error} (info {st.error_info:#x})"
     check_mask_invariants(mask, spec, block_q=kw.get("block_q"), block_k=kw.get("block_k"), causal=kw.get("causal", True))
     p = oracle_problem(spec, **kw)
     ora = so.build_mask_rows(p, w.q, w.k, rows, score_cache=score_cache, want_scores=True)
@@ -49,8 +51,7 @@ def assert_mask_parity(S, w, rows, *, impl="auto", score_cache=True, **kw):
     fin = np.isfinite(ora["scores"][same])
     np.testing.assert_allclose(sc[same][fin], ora["scores"][same][fin], rtol=2e-5, atol=2e-5)
     assert (sc[same][~fin] == -np.inf).all()
-    st = res.stats()
-    assert st.rows == flat.shape[0] and st.error == 0
+    assert st.rows == flat.shape[0]
     if rows is None:
         agree = same & (ora["min_gap"] >= 1e-5)
         if agree.all():

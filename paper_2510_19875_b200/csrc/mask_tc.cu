@@ -36,10 +36,13 @@ constexpr int kStageBytes = 4 * kHalfTile;     // [2 channel halves][2 tiles]
 constexpr int kQBytes = 2 * kR * kHalfTile;    // [2 channel halves][kR rows]
 constexpr int kMaxJobs = 64;
 constexpr int kListReaders = 1 + kMmaWarps + 4;  // producer warp, MMA warps, epilogue warps
-// A parity wait only means something to a thread that saw the phase before it complete. Chain c
-// goes to warp c % kMmaWarps and slot c % kSlots, so with this a warp is the only issuer that
-// ever waits on its slots and meets every phase of them.
-static_assert(kSlots % kMmaWarps == 0, "each TMEM slot must always meet the same issuing warp");
+// A parity wait only means something to a thread that saw the phase before it complete, and an
+// arrival only if it cannot come a phase early. So every stage buffer and every TMEM slot
+// belongs to one issuing warp: stage s of the kernel's whole sequence goes, with all its chains,
+// to warp s % kMmaWarps and lands in buffer s % kStages (the same number), and a warp's chains
+// alternate between its own two slots. The other issuing warps touch none of its barriers.
+static_assert(kStages == kMmaWarps, "a stage buffer must always meet the same issuing warp");
+static_assert(kSlots == 2 * kMmaWarps, "two private TMEM slots per issuing warp");
 
 struct Tail {
     unsigned long long full[kStages], empty[kStages], tmem_full[kSlots], tmem_empty[kSlots];
@@ -141,16 +144,16 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
     }
 }
 
-// kMmaWarps warps issue the chains in turn (chain c belongs to warp c % kMmaWarps): the waits,
-// commits and bookkeeping between two chains of one warp take several times longer than the
-// tensor core needs for a chain, so one issuing warp would leave it idle most of the time. All
-// issuing warps walk the same unit order; each is run by all 32 lanes, converged: warp-wide
-// waits, one elected lane issues.
+// kMmaWarps warps take the stages in turn (stage s belongs, with all its chains, to warp
+// s % kMmaWarps): the waits, commits and bookkeeping between two chains of one warp take several
+// times longer than the tensor core needs for a chain, so one issuing warp would leave it idle
+// most of the time. All issuing warps walk the same unit order; each is run by all 32 lanes,
+// converged: warp-wide waits, one elected lane issues.
 __device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_smem, unsigned tmem_base, int which) {
     const Geom &g = P.g;
-    Ring st, sl;
     unsigned grp_par = 0, q_par = 0, jr_par[kR] = {0, 0, 0, 0};
-    unsigned chain = 0;
+    unsigned stage_seq = 0;   // stages so far, over the whole kernel (the same in every role)
+    unsigned my_chains = 0;   // chains this warp has issued
     const unsigned q_lo = desc_lo_sw128(q_smem, 16);
     for (;;) {
         if (!mbar_wait_w(smem_u32(&tl->jobs_ready[kR]), grp_par, tl, P.ws, 201)) return;
@@ -171,21 +174,17 @@ __device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_
                 __syncwarp();
                 if (elect_one()) mbar_arrive(smem_u32(&tl->jobs_ack[li]));  // the count is all this role reads
                 __syncwarp();
-                for (int j = 0; j < n; j += 2) {
-                    const int r0 = level == 0 ? 0 : x, r1 = level == 0 ? R : x + 1;
-                    // Every issuing warp waits for every stage, with or without a chain in it: it
-                    // then sees each phase of full[] in turn (a warp that skipped some could take a
-                    // phase still in flight for the one after it), and its arrival on empty[] cannot
-                    // come before the stage's previous use was released.
-                    if (!mbar_wait_w(smem_u32(&tl->full[st.idx]), st.phase, tl, P.ws, 204)) return;
-                    bool issued = false;
-                    const unsigned a_lo = desc_lo_sw128(k_smem + st.idx * kStageBytes, 16);
-                    for (int r = r0; r < r1; ++r, ++chain, sl.advance(kSlots)) {
-                        if ((int)(chain % kMmaWarps) != which) continue;
-                        issued = true;
-                        if (!mbar_wait_w(smem_u32(&tl->tmem_empty[sl.idx]), sl.phase ^ 1, tl, P.ws, 205)) return;
+                const int r0 = level == 0 ? 0 : x, r1 = level == 0 ? R : x + 1;
+                for (int j = 0; j < n; j += 2, ++stage_seq) {
+                    if ((int)(stage_seq % kMmaWarps) != which) continue;  // another warp's stage: nothing to do
+                    const int sidx = which;  // = stage_seq % kStages
+                    if (!mbar_wait_w(smem_u32(&tl->full[sidx]), (stage_seq / kStages) & 1u, tl, P.ws, 204)) return;
+                    const unsigned a_lo = desc_lo_sw128(k_smem + sidx * kStageBytes, 16);
+                    for (int r = r0; r < r1; ++r, ++my_chains) {
+                        const int slot = 2 * which + (int)(my_chains & 1u);
+                        if (!mbar_wait_w(smem_u32(&tl->tmem_empty[slot]), ((my_chains >> 1) & 1u) ^ 1u, tl, P.ws, 205)) return;
                         tc_fence_after();
-                        const unsigned d_tmem = tmem_base + sl.idx * 64;
+                        const unsigned d_tmem = tmem_base + slot * 64;
                         const unsigned b_lo = q_lo + r * (kHalfTile >> 4);
                         if (elect_one()) {
 #pragma unroll
@@ -194,18 +193,13 @@ __device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_
                                 for (int k4 = 0; k4 < 4; ++k4)
                                     tc_mma_bf16_split(d_tmem, a_lo + ((c * 2 * kHalfTile + k4 * 32) >> 4), kDescHi,
                                                       b_lo + ((c * kR * kHalfTile + k4 * 32) >> 4), kDescHi, kIdesc, (c | k4) != 0);
-                            tc_commit(smem_u32(&tl->tmem_full[sl.idx]));
+                            tc_commit(smem_u32(&tl->tmem_full[slot]));
+                            // the stage is free once its last chain has read it (a commit covers all
+                            // earlier instructions of this thread)
+                            if (r + 1 == r1) tc_commit(smem_u32(&tl->empty[sidx]));
                         }
                         __syncwarp();
                     }
-                    // the stage is free once every issuing warp is done with it: those that read it
-                    // commit behind their chains, the others just arrive
-                    if (elect_one()) {
-                        if (issued) tc_commit(smem_u32(&tl->empty[st.idx]));
-                        else mbar_arrive(smem_u32(&tl->empty[st.idx]));
-                    }
-                    __syncwarp();
-                    st.advance(kStages);
                 }
             }
         }
@@ -214,8 +208,9 @@ __device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_
 
 __device__ void epilogue_role(const Params &P, Tail *tl, unsigned tmem_base, int wq, int lane) {
     const Geom &g = P.g;
-    Ring sl;
     unsigned grp_par = 0, jr_par[kR] = {0, 0, 0, 0};
+    unsigned stage_seq = 0;
+    unsigned chains = 0;  // chains each issuing warp has produced so far, mod 4: two bits per warp
     const int tile = wq >> 1;                // which tile of the pair this warp's lanes hold
     const int key = (wq & 1) * 32 + lane;    // key index inside the tile
     for (;;) {
@@ -234,15 +229,20 @@ __device__ void epilogue_role(const Params &P, Tail *tl, unsigned tmem_base, int
                     jr_par[x] ^= 1;
                 }
                 const int n = tl->n_jobs[li];
-                for (int j = 0; j < n; j += 2) {
+                for (int j = 0; j < n; j += 2, ++stage_seq) {
                     const int c = j + tile;
                     const int blk = c < n ? tl->jobs_blk[li][c] : -1;
                     const int r0 = level == 0 ? 0 : x, r1 = level == 0 ? R : x + 1;
+                    const int owner = (int)(stage_seq % kMmaWarps);
                     for (int r = r0; r < r1; ++r) {
-                        if (!mbar_wait(smem_u32(&tl->tmem_full[sl.idx]), sl.phase, tl, P.ws, 303)) return;
+                        // the owner's chains alternate between its two slots
+                        const unsigned cnt = (chains >> (2 * owner)) & 3u;
+                        const int slot = 2 * owner + (int)(cnt & 1u);
+                        chains = (chains & ~(3u << (2 * owner))) | (((cnt + 1u) & 3u) << (2 * owner));
+                        if (!mbar_wait(smem_u32(&tl->tmem_full[slot]), cnt >> 1, tl, P.ws, 303)) return;
                         tc_fence_after();
                         if (blk >= 0) {
-                            const unsigned taddr = tmem_base + sl.idx * 64 + ((unsigned)(wq * 32) << 16);
+                            const unsigned taddr = tmem_base + slot * 64 + ((unsigned)(wq * 32) << 16);
                             float v[64];
                             tmem_ld_32x32(taddr, v);
                             tmem_ld_32x32(taddr + 32, v + 32);
@@ -264,8 +264,7 @@ __device__ void epilogue_role(const Params &P, Tail *tl, unsigned tmem_base, int
                         }
                         tc_fence_before();
                         __syncwarp();
-                        if (lane == 0) mbar_arrive(smem_u32(&tl->tmem_empty[sl.idx]));
-                        sl.advance(kSlots);
+                        if (lane == 0) mbar_arrive(smem_u32(&tl->tmem_empty[slot]));
                     }
                 }
                 // this list is done for rows r0..r1: tell the controller
@@ -416,7 +415,7 @@ mask_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < kStages; ++i) { mbar_init(smem_u32(&tl->full[i]), 1); mbar_init(smem_u32(&tl->empty[i]), kMmaWarps); }
+        for (int i = 0; i < kStages; ++i) { mbar_init(smem_u32(&tl->full[i]), 1); mbar_init(smem_u32(&tl->empty[i]), 1); }
         for (int i = 0; i < kSlots; ++i) { mbar_init(smem_u32(&tl->tmem_full[i]), 1); mbar_init(smem_u32(&tl->tmem_empty[i]), 4); }
         mbar_init(smem_u32(&tl->q_full), 1);
         for (int i = 0; i <= kR; ++i) { mbar_init(smem_u32(&tl->jobs_ready[i]), 1); mbar_init(smem_u32(&tl->jobs_ack[i]), kListReaders); }

@@ -262,6 +262,64 @@ int so_build_mask_rows(const so_problem *p, const void *Q, const void *K, const 
 }
 
 /*
+ * Algorithm 2 with a sparsity constant of its own for every query block (the "variable k" the
+ * paper's discussion of needle depth and its fourth limitation name as the remedy for the
+ * stronger pruning of late rows; the paper leaves it undefined, so this is a reading): row
+ * (b, h, q) is the unchanged algorithm run with k = k_row[q], clamped to 1 .. k_top. Rows are
+ * k_top wide: the row's k entries, then -1 / -inf padding. Other arguments as above.
+ */
+int so_build_mask_rows_var(const so_problem *p, const void *Q, const void *K, const int32_t *k_row,
+                           const int64_t *rows, int64_t n_rows, int32_t *mask_out, float *score_out,
+                           float *min_gap_out, int64_t *tiles_out, int flags) {
+    int rc = check_problem(p);
+    if (rc) return rc;
+    if (!k_row) return -2;
+    const int64_t Nq = so_num_query_blocks(p), total = so_num_rows(p);
+    int err = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t i = 0; i < n_rows; ++i) {
+        int64_t id = rows ? rows[i] : i;
+        if (id < 0 || id >= total) { err = -3; continue; }
+        int64_t q = id % Nq, h = (id / Nq) % p->n_q_heads, b = id / Nq / p->n_q_heads;
+        so_problem pq = *p; /* the same problem with this row's k */
+        pq.k_top = k_row[q] < 1 ? 1 : (k_row[q] > p->k_top ? p->k_top : k_row[q]);
+        int32_t *m = malloc(sizeof(int32_t) * pq.k_top);
+        float *sc = score_out ? malloc(sizeof(float) * pq.k_top) : NULL;
+        if (!m || (score_out && !sc)) { err = -1; free(m); free(sc); continue; }
+        if (stream_row(&pq, Q, K, b, h, q, -1, flags, m, sc, min_gap_out ? min_gap_out + i : NULL,
+                       tiles_out ? tiles_out + i : NULL))
+            err = -1;
+        for (int64_t j = 0; j < p->k_top; ++j) {
+            mask_out[i * p->k_top + j] = j < pq.k_top ? m[j] : -1;
+            if (score_out) score_out[i * p->k_top + j] = j < pq.k_top ? sc[j] : -INFINITY;
+        }
+        free(m); free(sc);
+    }
+    return err;
+}
+
+/*
+ * A schedule for k_row: the effective-sparsity formula of the needle-depth experiment,
+ * k = floor(1 + (n - 1) s), applied to each query block with n = the number of key blocks that
+ * row may look at (the paper applies it once with n = T / b_q; taking the row's own count is
+ * what makes the pruning ratio the same from the top to the bottom of a causal pattern).
+ * Clamped to 1 .. k_top. k_row_out has ceil(T / b_q) entries.
+ */
+int so_k_schedule(const so_problem *p, double s, int32_t *k_row_out) {
+    int rc = check_problem(p);
+    if (rc) return rc;
+    if (!(s > 0.0 && s < 1.0)) return -2;
+    const int64_t Nq = so_num_query_blocks(p), N_k = padded_len(p) / p->block_k;
+    for (int64_t q = 0; q < Nq; ++q) {
+        int64_t n = 0;
+        for (int64_t r = 0; r < N_k; ++r) n += c_blk(p, q, r);
+        int64_t k = (int64_t)floor(1.0 + (double)(n - 1) * s);
+        k_row_out[q] = (int32_t)(k < 1 ? 1 : (k > p->k_top ? p->k_top : k));
+    }
+    return 0;
+}
+
+/*
  * Eq. 2 on block masks: for every query token of each listed row, softmax over the keys of the
  * row's selected blocks that C allows, then the weighted sum of V, all in fp64.
  *   mask [n_rows, k]  as produced above; out [n_rows, b_q, d] fp64; tokens beyond T or with no

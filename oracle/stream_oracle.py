@@ -101,6 +101,11 @@ def _load():
         lib.so_build_mask_rows.restype = ctypes.c_int
         lib.so_build_mask_rows.argtypes = [ctypes.POINTER(_CProblem), vp, vp, i64p, ctypes.c_int64,
                                            vp, vp, vp, vp, ctypes.c_int, ctypes.c_int]
+        lib.so_build_mask_rows_var.restype = ctypes.c_int
+        lib.so_build_mask_rows_var.argtypes = [ctypes.POINTER(_CProblem), vp, vp, vp, i64p, ctypes.c_int64,
+                                               vp, vp, vp, vp, ctypes.c_int]
+        lib.so_k_schedule.restype = ctypes.c_int
+        lib.so_k_schedule.argtypes = [ctypes.POINTER(_CProblem), ctypes.c_double, vp]
         lib.so_sparse_attention_rows.restype = ctypes.c_int
         lib.so_sparse_attention_rows.argtypes = [ctypes.POINTER(_CProblem), vp, vp, vp, i64p, ctypes.c_int64,
                                                  vp, ctypes.c_double, vp]
@@ -162,6 +167,42 @@ def build_mask_rows(p: OracleProblem, q: np.ndarray, k: np.ndarray, rows=None, *
     out = {"mask": mask, "min_gap": gap, "tiles": tiles}
     if want_scores:
         out["scores"] = scores
+    return out
+
+
+def build_mask_rows_var(p: OracleProblem, q: np.ndarray, k: np.ndarray, k_row: np.ndarray, rows=None, *,
+                        score_cache: bool = False, want_scores: bool = False):
+    """Algorithm 2 with ``k = k_row[query block]`` per row (clamped to 1 .. k_top); same returns as
+    :func:`build_mask_rows`, rows ``k_top`` wide."""
+    _check(p, q, p.n_q_heads, "q"), _check(p, k, p.n_kv_heads, "k")
+    lib = _load()
+    k_row = np.ascontiguousarray(k_row, dtype=np.int32)
+    if k_row.shape != (num_query_blocks(p),):
+        raise ValueError(f"k_row: need shape {(num_query_blocks(p),)}, got {k_row.shape}")
+    rows_arr = None if rows is None else np.ascontiguousarray(rows, dtype=np.int64)
+    n = num_rows(p) if rows_arr is None else rows_arr.shape[0]
+    mask = np.empty((n, p.k_top), np.int32)
+    gap = np.empty((n,), np.float32)
+    tiles = np.empty((n,), np.int64)
+    scores = np.empty((n, p.k_top), np.float32) if want_scores else None
+    rc = lib.so_build_mask_rows_var(ctypes.byref(p.c()), _ptr(q), _ptr(k), _ptr(k_row), _ptr(rows_arr), n,
+                                    _ptr(mask), _ptr(scores), _ptr(gap), _ptr(tiles),
+                                    SCORE_CACHE if score_cache else 0)
+    if rc:
+        raise RuntimeError(f"so_build_mask_rows_var failed with {rc}")
+    out = {"mask": mask, "min_gap": gap, "tiles": tiles}
+    if want_scores:
+        out["scores"] = scores
+    return out
+
+
+def k_schedule(p: OracleProblem, s: float) -> np.ndarray:
+    """``k`` per query block from the effective sparsity ``s`` (0 < s < 1) and the row's own number
+    of allowed key blocks; int32 [ceil(T / block_q)], clamped to 1 .. k_top."""
+    out = np.empty((num_query_blocks(p),), np.int32)
+    rc = _load().so_k_schedule(ctypes.byref(p.c()), float(s), _ptr(out))
+    if rc:
+        raise RuntimeError(f"so_k_schedule failed with {rc}")
     return out
 
 

@@ -140,20 +140,25 @@ def test_hand_example():
         line = line.strip()
         if not line or line.startswith("#"):
             continue
-        if line == "case":
+        if line in ("case", "case_var"):
             cur = {"rows": {}}
             cases.append(cur)
+        elif line.startswith("k_row:"):
+            cur["k_row"] = [int(x) for x in line[6:].split()]
         elif line.startswith("K:"):
             cur["K"] = [float(x) for x in line[2:].split()]
         else:
             qb, vals = line.split(":")
             cur["rows"][int(qb)] = [int(x) for x in vals.split()]
-    assert len(cases) == 2
+    assert len(cases) == 3 and sum("k_row" in c for c in cases) == 1
     for c in cases:
         K = np.array(c["K"], np.float32).reshape(1, 1, 8, 1)
         Q = np.ones((1, 1, 8, 1), np.float32)
         p = so.OracleProblem(1, 1, 1, 8, 1, 1, 1, 2, True, "f32")
-        mask = so.build_mask_rows(p, Q, K)["mask"]
+        if "k_row" in c:
+            mask = so.build_mask_rows_var(p, Q, K, np.array(c["k_row"], np.int32))["mask"]
+        else:
+            mask = so.build_mask_rows(p, Q, K)["mask"]
         for qb, want in c["rows"].items():
             assert mask[qb].tolist() == want
 
@@ -401,3 +406,62 @@ def test_mask_difference_is_the_row_wise_set_difference():
         assert dsc[i][: len(kept)].tolist() == [float(sc[i][a[i].tolist().index(x)]) for x in want]
     d, _ = so.mask_difference(np.array([[0, 3, 5, 9, -1, -1]], np.int32), np.array([[0, 9, -1]], np.int32))
     assert d.tolist() == [[3, 5, -1, -1, -1, -1]]
+
+
+@pytest.mark.parametrize("case", RANDOM_CASES[:8])
+def test_variable_k_rows_match_independent_simulation(case):
+    """Each row of the variable-k build is Algorithm 2 with that row's own k: checked against the
+    list-based simulation above, run with the row's k, on k_row values that include 1, k_top and
+    out-of-range entries (clamped)."""
+    import dataclasses
+
+    B, H, G, T, d, bq, bk, k, causal, dtype = case
+    rng = np.random.default_rng(hash(case) % (2**32) + 1)
+    q = grid_inputs(rng, (B, H, T, d), dtype, 1 / 16)
+    kk = grid_inputs(rng, (B, G, T, d), dtype, 1 / 16)
+    p = so.OracleProblem(B, H, G, T, d, bq, bk, k, causal, dtype)
+    nq_rows = so.num_query_blocks(p)
+    k_row = rng.integers(1, k + 1, size=nq_rows).astype(np.int32)
+    k_row[0], k_row[-1] = 0, k + 3  # clamped to 1 and k
+    if nq_rows > 3:
+        k_row[1], k_row[2] = 1, k
+    got = so.build_mask_rows_var(p, q, kk, k_row, want_scores=True)
+    assert got["mask"].shape == (B * H * nq_rows, k)
+    for b in range(B):
+        for h in range(H):
+            table, _, nk = block_score_table(p, q, kk, b, h)
+            for qb in range(nq_rows):
+                kq = int(min(max(k_row[qb], 1), k))
+                kept, scored, _ = simulate_row(dataclasses.replace(p, k_top=kq), table, nk, qb)
+                i = (b * H + h) * nq_rows + qb
+                assert got["mask"][i].tolist() == padded(kept, k), (case, b, h, qb, kq)
+                assert got["tiles"][i] == len(scored)
+                assert got["scores"][i, : len(kept)].tolist() == [float(table[qb, r]) for r in kept]
+                assert np.isneginf(got["scores"][i, len(kept):]).all()
+
+
+def test_variable_k_with_constant_schedule_is_the_fixed_k_build():
+    rng = np.random.default_rng(11)
+    p = so.OracleProblem(1, 2, 1, 96, 4, 4, 4, 3, True, "f32")
+    q = grid_inputs(rng, (1, 2, 96, 4), "f32")
+    k = grid_inputs(rng, (1, 1, 96, 4), "f32")
+    a = so.build_mask_rows(p, q, k, want_scores=True)
+    b = so.build_mask_rows_var(p, q, k, np.full(so.num_query_blocks(p), 3, np.int32), want_scores=True)
+    for key in ("mask", "scores", "min_gap", "tiles"):
+        np.testing.assert_array_equal(a[key], b[key])
+
+
+@pytest.mark.parametrize("causal", [True, False])
+def test_k_schedule_closed_form(causal):
+    """k(q) = floor(1 + (n(q) - 1) s) with n(q) the row's allowed key blocks: q + 1 under a causal
+    mask with equal blocks, all of them without one; clamped to k_top."""
+    T, blk, k_top, s = 64 * 4 - 3, 4, 12, 0.25
+    p = so.OracleProblem(1, 1, 1, T, 2, blk, blk, k_top, causal, "f32")
+    got = so.k_schedule(p, s)
+    nq = -(-T // blk)
+    n = np.arange(1, nq + 1) if causal else np.full(nq, nq)
+    want = np.clip(np.floor(1 + (n - 1) * s), 1, k_top).astype(np.int32)
+    assert got.tolist() == want.tolist()
+    assert got.max() == k_top and (not causal or got[0] == 1)  # the clamp is reached
+    with pytest.raises(RuntimeError):
+        so.k_schedule(p, 1.0)

@@ -42,6 +42,8 @@ def parse_args():
     ap.add_argument("--workload", default="cot_layer_128k")
     ap.add_argument("--T", type=int, default=0, help="override the workload's context length")
     ap.add_argument("--kernels", default="auto", choices=["auto", "generic", "tensor"], help="library kernel choice")
+    ap.add_argument("--k-sparsity", type=float, default=0.0,
+                    help="build the mask with k per query block from this effective sparsity (0 = one k; implies --no-e2e)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="target CPU time of the oracle sample")
@@ -272,9 +274,19 @@ def run_ours(args):
     out = torch.empty_like(q)
     ws = S.new_workspace(p, dev)
     stream = torch.cuda.current_stream()
+    k_row = None
+    if args.k_sparsity > 0:
+        k_row = S.k_schedule(p, args.k_sparsity).to(dev)
+        args.no_e2e = True  # the host entry point takes one k
+
+    def build_mask():
+        if k_row is None:
+            S.stream_build_mask(p, q, k, mask, None, ws, ws.numel(), stream)
+        else:
+            S.stream_build_mask_var(p, q, k, k_row, mask, None, ws, ws.numel(), stream)
 
     def step():
-        S.stream_build_mask(p, q, k, mask, None, ws, ws.numel(), stream)
+        build_mask()
         S.stream_sparse_attention(p, q, k, v, mask, 0.0, out, stream)
 
     for _ in range(args.warmup):
@@ -290,7 +302,7 @@ def run_ours(args):
     t_begin.record()
     for i in range(args.steps):
         ev[i][0].record()
-        S.stream_build_mask(p, q, k, mask, None, ws, ws.numel(), stream)
+        build_mask()
         ev[i][1].record()
         S.stream_sparse_attention(p, q, k, v, mask, 0.0, out, stream)
         ev[i][2].record()
@@ -366,11 +378,13 @@ def run_ours(args):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": spec.dtype, "data": "synthetic",
         "config": workload_config(spec, {"l2": "inputs larger than L2 (Q+K+V %.0f MiB per step)" % (
-            (q.numel() + 2 * k.numel()) * esz / 2**20), "kernels": args.kernels, "per_rank": "one independent layer each"}),
+            (q.numel() + 2 * k.numel()) * esz / 2**20), "kernels": args.kernels, "per_rank": "one independent layer each",
+            **({"k_schedule": {"effective_sparsity": args.k_sparsity, "k_min": int(k_row.min()), "k_max": int(k_row.max()),
+                               "k_mean": float(k_row.float().mean())}} if k_row is not None else {})}),
         "mask_build": kernels["stream_build_mask"], "sparse_attention": kernels["stream_sparse_attention"],
         "roofline": {"kernel": dom["kernel"], "entry_point": dominant, "bound": "hbm", "achieved": dom["algorithmic_gbs"],
                      "peak": peak, "unit": "GB/s", "frac": dom["algorithmic_gbs"] / peak,
-                     "traffic": ncu_traffic(dom["kernel"], spec) if dom["kernel"] in KERNEL_SOURCES else None,
+                     "traffic": ncu_traffic(dom["kernel"], spec) if dom["kernel"] in KERNEL_SOURCES and k_row is None else None,
                      "peak_kind": f"of {peak_kind}", "algorithmic_bytes": dom["algorithmic_bytes"],
                      "share_of_step": dom["ms"] / (mask_ms + attn_ms),
                      "frac_of_8TBs_nominal": dom["algorithmic_gbs"] / 8000.0},

@@ -110,6 +110,35 @@ stream_status stream_build_mask(const stream_problem *p, const void *q, const vo
                                 float *score_out, void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * stream_build_mask with a sparsity constant of its own for every query block ("variable k": the
+ * paper's discussion of needle depth, Section 4.2, and the fourth item of its Limitations name it
+ * as the remedy for the stronger pruning of late rows under a causal mask, and leave it
+ * undefined). The reading taken: the row of query block qb is Algorithm 2, unchanged, run with
+ * k = k_row[qb]; rows stay k_top wide (the row's blocks ascending, then -1; scores -inf padded),
+ * so the result feeds stream_sparse_attention, stream_vertical_scores and stream_mask_difference
+ * as it is.
+ *
+ *   k_row      device int32 [ceil(T/block_q)], shared by all heads and batch entries; read only.
+ *              Entries outside 1 .. k_top are clamped into that range.
+ * Everything else as stream_build_mask (p->k_top is the row width and the largest k).
+ */
+stream_status stream_build_mask_var(const stream_problem *p, const void *q, const void *k, const int32_t *k_row,
+                                    int32_t *mask_out, float *score_out, void *workspace, size_t workspace_bytes,
+                                    void *cuda_stream);
+
+/*
+ * A schedule for stream_build_mask_var, computed on the host: the effective-sparsity formula of
+ * Section 4.2, k = floor(1 + (n - 1) s), applied per query block with n = the number of key
+ * blocks that row may look at (qb + 1 blocks under a causal mask with equal block sizes; the
+ * paper applies the formula once, with n = T / b_q, which is what prunes late rows harder).
+ * Clamped to 1 .. p->k_top.
+ *
+ *   s           0 < s < 1, else INVALID_ARG
+ *   k_row_host  HOST int32 [ceil(T/block_q)], overwritten; copy it to the device for the build
+ */
+stream_status stream_k_schedule(const stream_problem *p, double s, int32_t *k_row_host);
+
+/*
  * stream_build_mask without a caller-provided workspace and without any allocation. (The paper
  * has no counterpart to this entry point; it exists for deployment.)
  *

@@ -1,4 +1,5 @@
 // extern "C" boundary of libstream: argument validation, geometry, dispatch. See stream.h.
+#include <cmath>
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
@@ -61,13 +62,8 @@ stream_status make_geom(const stream_problem *p, Geom *g) {
     g->batch = p->batch; g->H = p->n_q_heads; g->G = p->n_kv_heads; g->hpg = p->n_q_heads / p->n_kv_heads;
     g->T = p->T; g->d = p->d; g->bq = p->block_q; g->bk = p->block_k; g->k_top = p->k_top; g->causal = p->causal;
     g->n_qb = (int)n_qb; g->N_k = (int)N_k;
-    // levels until every node is a single block: nodes start with at most ceil(N_k / k) blocks and
-    // the larger half of n blocks has ceil(n / 2). With N_k > 1 the first level always runs (it is
-    // where scores are first computed), matching n_it = ceil(log2 N_k) >= 1.
-    long long sz = (N_k + p->k_top - 1) / p->k_top;
-    int levels = 0;
-    while (sz > 1) { sz = (sz + 1) / 2; ++levels; }
-    g->levels = N_k > 1 ? (levels > 1 ? levels : 1) : 0;
+    g->levels = levels_for((int)N_k, p->k_top);
+    g->k_row = nullptr;
     g->qs_b = p->q_stride_b; g->qs_h = p->q_stride_h; g->qs_t = p->q_stride_t;
     g->ks_b = p->kv_stride_b; g->ks_h = p->kv_stride_h; g->ks_t = p->kv_stride_t;
     return STREAM_OK;
@@ -142,11 +138,14 @@ size_t stream_workspace_bytes(const stream_problem *p) {
     return sizeof(WorkspaceHeader);
 }
 
-stream_status stream_build_mask(const stream_problem *p, const void *q, const void *k, int32_t *mask_out,
-                                float *score_out, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+// Both mask entry points: k_row == NULL is the fixed-k build.
+static stream_status build_mask_impl(const stream_problem *p, const void *q, const void *k, const int32_t *k_row,
+                                     int32_t *mask_out, float *score_out, void *workspace, size_t workspace_bytes,
+                                     void *cuda_stream) {
     Geom g;
     stream_status rc = make_geom(p, &g);
     if (rc != STREAM_OK) return rc;
+    g.k_row = k_row;
     if (q == nullptr || k == nullptr || mask_out == nullptr) { set_error("q, k and mask_out must not be NULL"); return STREAM_ERR_INVALID_ARG; }
     if (workspace == nullptr || workspace_bytes < sizeof(WorkspaceHeader) || ((uintptr_t)workspace & 255) != 0) {
         set_error("workspace must be a 256-byte aligned device buffer of at least %zu bytes", sizeof(WorkspaceHeader));
@@ -163,6 +162,32 @@ stream_status stream_build_mask(const stream_problem *p, const void *q, const vo
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(workspace)");
     if (tc_ok && p->impl != STREAM_IMPL_GENERIC) return launch_mask_tc(g, q, k, mask_out, score_out, ws, st);
     return launch_mask_generic(g, p->dtype, q, k, mask_out, score_out, ws, st);
+}
+
+stream_status stream_build_mask(const stream_problem *p, const void *q, const void *k, int32_t *mask_out,
+                                float *score_out, void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    return build_mask_impl(p, q, k, nullptr, mask_out, score_out, workspace, workspace_bytes, cuda_stream);
+}
+
+stream_status stream_build_mask_var(const stream_problem *p, const void *q, const void *k, const int32_t *k_row,
+                                    int32_t *mask_out, float *score_out, void *workspace, size_t workspace_bytes,
+                                    void *cuda_stream) {
+    if (k_row == nullptr) { set_error("k_row must not be NULL (use stream_build_mask for one k)"); return STREAM_ERR_INVALID_ARG; }
+    return build_mask_impl(p, q, k, k_row, mask_out, score_out, workspace, workspace_bytes, cuda_stream);
+}
+
+stream_status stream_k_schedule(const stream_problem *p, double s, int32_t *k_row_host) {
+    Geom g;
+    stream_status rc = make_geom(p, &g);
+    if (rc != STREAM_OK) return rc;
+    if (k_row_host == nullptr) { set_error("k_row_host must not be NULL"); return STREAM_ERR_INVALID_ARG; }
+    if (!(s > 0.0 && s < 1.0)) { set_error("effective sparsity must lie strictly between 0 and 1 (got %g)", s); return STREAM_ERR_INVALID_ARG; }
+    for (int qb = 0; qb < g.n_qb; ++qb) {
+        const long long n = (long long)last_valid_block(g, qb) + 1;  // key blocks the row may look at
+        long long kq = (long long)floor(1.0 + (double)(n - 1) * s);
+        k_row_host[qb] = (int32_t)(kq < 1 ? 1 : (kq > g.k_top ? g.k_top : kq));
+    }
+    return STREAM_OK;
 }
 
 stream_status stream_sparse_attention(const stream_problem *p, const void *q, const void *k, const void *v,

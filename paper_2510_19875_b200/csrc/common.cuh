@@ -15,7 +15,8 @@ struct Geom {
     int d, bq, bk, k_top, causal;
     int n_qb;                   // ceil(T / bq): rows per head
     int N_k;                    // key blocks after padding T to a multiple of lcm(bq, bk)
-    int levels;                 // split levels that can change the result
+    int levels;                 // split levels that can change the result (with k = k_top)
+    const int32_t *k_row;       // device, [n_qb]: k of each query block (clamped to 1 .. k_top), or NULL = k_top everywhere
     long long qs_b, qs_h, qs_t; // element strides
     long long ks_b, ks_h, ks_t;
 };
@@ -57,6 +58,23 @@ stream_status read_attn_status(unsigned int out[2], cudaStream_t st);
 
 __device__ __forceinline__ float to_float(float x) { return x; }
 __device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+// Levels until every node is a single block: nodes start with at most ceil(N_k / k) blocks and
+// the larger half of n blocks has ceil(n / 2). With N_k > 1 the first level always runs (it is
+// where scores are first computed), matching n_it = ceil(log2 N_k) >= 1.
+__host__ __device__ inline int levels_for(int N_k, int k) {
+    long long sz = ((long long)N_k + k - 1) / k;
+    int levels = 0;
+    while (sz > 1) { sz = (sz + 1) / 2; ++levels; }
+    return N_k > 1 ? (levels > 1 ? levels : 1) : 0;
+}
+
+// The sparsity constant of query block qb.
+__device__ __forceinline__ int row_k(const Geom &g, int qb) {
+    if (g.k_row == nullptr) return g.k_top;
+    const int k = g.k_row[qb];
+    return k < 1 ? 1 : (k > g.k_top ? g.k_top : k);
+}
 
 // Last key block a row may look at (C^blk of Algorithm 2 in closed form), -1 if none.
 __host__ __device__ inline int last_valid_block(const Geom &g, int qb) {

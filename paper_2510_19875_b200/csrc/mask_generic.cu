@@ -90,6 +90,8 @@ __global__ void __launch_bounds__(kThreads) mask_generic_kernel(Geom g, const T 
     const T *qp = q + b * g.qs_b + h * g.qs_h;
     const T *kp = k + b * g.ks_b + kvh * g.ks_h;
     const int q_lim = last_valid_block(g, qb);
+    const int kq = row_k(g, qb);  // this row's k (= k_top unless a schedule was given)
+    const int levels = g.k_row == nullptr ? g.levels : levels_for(g.N_k, kq);
 
     for (int idx = tid; idx < kTile * D; idx += kThreads) {
         int m = idx / D, c = idx % D;
@@ -98,9 +100,9 @@ __global__ void __launch_bounds__(kThreads) mask_generic_kernel(Geom g, const T 
     }
     if (tid == 0) {  // initial nodes tiling [0, N_k); keep those that hold an allowed block
         int n = 0;
-        for (int j = 0; j < g.k_top; ++j) {
-            int f = (int)(((long long)j * g.N_k) / g.k_top);
-            int l = (int)(((long long)(j + 1) * g.N_k) / g.k_top) - 1;
+        for (int j = 0; j < kq; ++j) {
+            int f = (int)(((long long)j * g.N_k) / kq);
+            int l = (int)(((long long)(j + 1) * g.N_k) / kq) - 1;
             if (f <= l && f <= q_lim) { node_f[n] = f; node_l[n] = l; node_s[n] = CUDART_NAN_F; ++n; }
         }
         s_nodes = n;
@@ -108,7 +110,7 @@ __global__ void __launch_bounds__(kThreads) mask_generic_kernel(Geom g, const T 
     __syncthreads();
 
     unsigned tiles = 0;
-    for (int level = 0; level < g.levels; ++level) {
+    for (int level = 0; level < levels; ++level) {
         if (tid == 0) {
             int n = 0;
             for (int i = 0; i < s_nodes; ++i) {
@@ -132,14 +134,14 @@ __global__ void __launch_bounds__(kThreads) mask_generic_kernel(Geom g, const T 
         // top-k by rank: a candidate is beaten by a higher score, or an equal score at a lower index
         for (int c = tid; c < n_cand; c += kThreads) {
             int rank = 0;
-            if (n_cand > g.k_top) {
+            if (n_cand > kq) {
                 float s = cand_s[c];
                 for (int u = 0; u < n_cand; ++u) {
                     float su = cand_s[u];
                     rank += (su > s) || (su == s && u < c);
                 }
             }
-            keep[c] = rank < g.k_top;
+            keep[c] = rank < kq;
         }
         __syncthreads();
         if (tid == 0) {  // survivors stay in ascending block order

@@ -56,6 +56,7 @@ struct Tail {
     unsigned int tmem_base;
     int abort_flag;
     int grp_id, grp_b, grp_kvh, grp_qb, grp_h0, grp_R;
+    int grp_levels;  // levels of this group's rows (they share the query block, hence k)
     int n_jobs[kR + 1];
     int jobs_blk[kR + 1][kMaxJobs];
     float part[kR][kMaxJobs][2];
@@ -103,6 +104,7 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
         grp_par ^= 1;
         if (tl->grp_id < 0) return;
         const int b = tl->grp_b, kvh = tl->grp_kvh, qb = tl->grp_qb, h0 = tl->grp_h0, R = tl->grp_R;
+        const int levels = tl->grp_levels;
         // Q tiles of the group's rows (previous group's MMAs are all complete by now)
         if (elect_one()) {
             mbar_arrive_expect_tx(smem_u32(&tl->q_full), (unsigned)(R * 2 * kHalfTile));
@@ -111,7 +113,7 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
                     tma_load_4d(q_smem + (c * kR + r) * kHalfTile, tq, smem_u32(&tl->q_full), c * 64, qb * kBlk, h0 + r, b);
         }
         __syncwarp();
-        for (int level = 0; level < g.levels; ++level) {
+        for (int level = 0; level < levels; ++level) {
             const int lists = level == 0 ? 1 : R;
             for (int x = 0; x < lists; ++x) {
                 const int li = level == 0 ? kR : x;
@@ -159,10 +161,10 @@ __device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_
         if (!mbar_wait_w(smem_u32(&tl->jobs_ready[kR]), grp_par, tl, P.ws, 201)) return;
         grp_par ^= 1;
         if (tl->grp_id < 0) return;
-        const int R = tl->grp_R;
+        const int R = tl->grp_R, levels = tl->grp_levels;
         if (!mbar_wait_w(smem_u32(&tl->q_full), q_par, tl, P.ws, 202)) return;
         q_par ^= 1;
-        for (int level = 0; level < g.levels; ++level) {
+        for (int level = 0; level < levels; ++level) {
             const int lists = level == 0 ? 1 : R;
             for (int x = 0; x < lists; ++x) {
                 const int li = level == 0 ? kR : x;
@@ -217,10 +219,10 @@ __device__ void epilogue_role(const Params &P, Tail *tl, unsigned tmem_base, int
         if (!mbar_wait(smem_u32(&tl->jobs_ready[kR]), grp_par, tl, P.ws, 301)) return;
         grp_par ^= 1;
         if (tl->grp_id < 0) return;
-        const int R = tl->grp_R, qb = tl->grp_qb;
+        const int R = tl->grp_R, qb = tl->grp_qb, levels = tl->grp_levels;
         const long long rem_q = g.T - (long long)qb * kBlk;
         const int m_lim = rem_q < kBlk ? (int)rem_q : kBlk;  // query tokens of this block inside T
-        for (int level = 0; level < g.levels; ++level) {
+        for (int level = 0; level < levels; ++level) {
             const int lists = level == 0 ? 1 : R;
             for (int x = 0; x < lists; ++x) {
                 const int li = level == 0 ? kR : x;
@@ -319,9 +321,12 @@ __device__ void controller_role(const Params &P, Tail *tl, int lane) {
             R = min(kR, g.hpg - chunk * kR);
         }
         const int q_lim = last_valid_block(g, qb);
+        // the group's k: all its rows are the same query block
+        const int kq = done ? g.k_top : row_k(g, qb);
+        const int levels = g.k_row == nullptr ? g.levels : levels_for(g.N_k, kq);
         // initial nodes: lane i holds node i (the same for every row of the group)
-        int f0 = (int)(((long long)lane * g.N_k) / g.k_top), l0 = (int)(((long long)(lane + 1) * g.N_k) / g.k_top) - 1;
-        const bool v0 = !done && lane < g.k_top && f0 <= l0 && f0 <= q_lim;
+        int f0 = (int)(((long long)lane * g.N_k) / kq), l0 = (int)(((long long)(lane + 1) * g.N_k) / kq) - 1;
+        const bool v0 = !done && lane < kq && f0 <= l0 && f0 <= q_lim;
         const int m0 = (f0 + l0) / 2;
         const bool vl1 = v0, vr1 = v0 && m0 + 1 <= l0 && m0 + 1 <= q_lim;
         const unsigned bl = __ballot_sync(0xffffffffu, vl1), br = __ballot_sync(0xffffffffu, vr1);
@@ -335,6 +340,7 @@ __device__ void controller_role(const Params &P, Tail *tl, int lane) {
         if (lane == 0) {
             tl->n_jobs[kR] = n1;
             tl->grp_id = done ? -1 : id; tl->grp_b = b; tl->grp_kvh = kvh; tl->grp_qb = qb; tl->grp_h0 = h0; tl->grp_R = R;
+            tl->grp_levels = levels;
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&tl->jobs_ready[kR]));
@@ -344,7 +350,7 @@ __device__ void controller_role(const Params &P, Tail *tl, int lane) {
         float ns[kR];
         bool has_r[kR];
         unsigned tiles = (unsigned)(n1 * R);
-        for (int level = 0; level < g.levels; ++level) {
+        for (int level = 0; level < levels; ++level) {
 #pragma unroll
             for (int r = 0; r < kR; ++r) {
                 if (r >= R) continue;
@@ -364,7 +370,7 @@ __device__ void controller_role(const Params &P, Tail *tl, int lane) {
                     sl = ns[r];
                     if (vr) sr = fmaxf(tl->part[r][my_c[r]][0], tl->part[r][my_c[r]][1]);
                 }
-                const Keep kp = select_topk(vl, sl, vr, sr, g.k_top, lane);
+                const Keep kp = select_topk(vl, sl, vr, sr, kq, lane);
                 const unsigned kl = __ballot_sync(0xffffffffu, kp.l), kr = __ballot_sync(0xffffffffu, kp.r);
                 const int pos_l = __popc(kl & lt) + __popc(kr & lt), pos_r = pos_l + (kp.l ? 1 : 0);
                 __syncwarp();
@@ -376,7 +382,7 @@ __device__ void controller_role(const Params &P, Tail *tl, int lane) {
                 nf[r] = live ? tl->node_f[lane] : 0;
                 nl[r] = live ? tl->node_l[lane] : -1;
                 ns[r] = live ? tl->node_s[lane] : -CUDART_INF_F;
-                if (level + 1 < g.levels) {
+                if (level + 1 < levels) {
                     // next level: only right branches need a tile; left ones keep the node's score
                     const int mm = (nf[r] + nl[r]) / 2;
                     has_r[r] = live && nl[r] > nf[r] && mm + 1 <= q_lim;

@@ -74,6 +74,10 @@ def _load():
     lib.stream_workspace_bytes.argtypes = [P]
     lib.stream_build_mask.restype = ctypes.c_int
     lib.stream_build_mask.argtypes = [P, vp, vp, vp, vp, vp, sz, vp]
+    lib.stream_build_mask_var.restype = ctypes.c_int
+    lib.stream_build_mask_var.argtypes = [P, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.stream_k_schedule.restype = ctypes.c_int
+    lib.stream_k_schedule.argtypes = [P, ctypes.c_double, vp]
     lib.stream_build_mask_static.restype = ctypes.c_int
     lib.stream_build_mask_static.argtypes = [P, vp, vp, vp, vp, vp]
     lib.stream_sparse_attention.restype = ctypes.c_int
@@ -131,6 +135,18 @@ def stream_workspace_bytes(p: StreamProblem) -> int:
 def stream_build_mask(p: StreamProblem, q, k, mask_out, score_out, workspace, workspace_bytes: int, stream=None) -> None:
     _raise(_load().stream_build_mask(ctypes.byref(p), _addr(q), _addr(k), _addr(mask_out), _addr(score_out),
                                      _addr(workspace), workspace_bytes, _stream_handle(stream)))
+
+
+def stream_build_mask_var(p: StreamProblem, q, k, k_row, mask_out, score_out, workspace, workspace_bytes: int,
+                          stream=None) -> None:
+    """Mask build with ``k = k_row[query block]`` (device int32 array) instead of one k."""
+    _raise(_load().stream_build_mask_var(ctypes.byref(p), _addr(q), _addr(k), _addr(k_row), _addr(mask_out),
+                                         _addr(score_out), _addr(workspace), workspace_bytes, _stream_handle(stream)))
+
+
+def stream_k_schedule(p: StreamProblem, s: float, k_row_host) -> None:
+    """Fills the HOST int32 array ``k_row_host`` ([ceil(T / block_q)]) with the per-row k for sparsity ``s``."""
+    _raise(_load().stream_k_schedule(ctypes.byref(p), float(s), _addr(k_row_host)))
 
 
 def stream_build_mask_static(p: StreamProblem, q, k, mask_out, score_out, stream=None) -> None:
@@ -217,7 +233,9 @@ def new_workspace(p: StreamProblem, device) -> torch.Tensor:
 
 def build_mask(q: torch.Tensor, k: torch.Tensor, *, block_q: int, block_k: int, k_top: int, causal: bool = True,
                impl: str = "auto", want_scores: bool = False, mask_out: torch.Tensor | None = None,
-               workspace: torch.Tensor | None = None, stream=None) -> MaskResult:
+               workspace: torch.Tensor | None = None, k_row: torch.Tensor | None = None, stream=None) -> MaskResult:
+    """Mask of every row. With ``k_row`` (int32 CUDA tensor, one k per query block, see
+    :func:`k_schedule`) each row uses its own k and ``k_top`` is the row width."""
     if not q.is_cuda or not k.is_cuda:
         raise ValueError("q and k must be CUDA tensors (there is no CPU path)")
     p = make_problem(q, k, block_q=block_q, block_k=block_k, k_top=k_top, causal=causal, impl=impl)
@@ -225,8 +243,22 @@ def build_mask(q: torch.Tensor, k: torch.Tensor, *, block_q: int, block_k: int, 
     mask = mask_out if mask_out is not None else torch.empty(shape, dtype=torch.int32, device=q.device)
     scores = torch.empty(shape, dtype=torch.float32, device=q.device) if want_scores else None
     ws = workspace if workspace is not None else new_workspace(p, q.device)
-    stream_build_mask(p, q, k, mask, scores, ws, ws.numel(), stream)
+    if k_row is None:
+        stream_build_mask(p, q, k, mask, scores, ws, ws.numel(), stream)
+    else:
+        if not k_row.is_cuda or k_row.dtype != torch.int32 or not k_row.is_contiguous() or tuple(k_row.shape) != (shape[2],):
+            raise ValueError(f"k_row must be a contiguous int32 CUDA tensor of shape ({shape[2]},)")
+        stream_build_mask_var(p, q, k, k_row, mask, scores, ws, ws.numel(), stream)
     return MaskResult(mask, scores, ws)
+
+
+def k_schedule(p: StreamProblem, s: float) -> torch.Tensor:
+    """Host int32 tensor [ceil(T / block_q)]: k per query block for an effective sparsity ``s``
+    (the formula of :func:`effective_k` applied to each row's own number of allowed key blocks,
+    clamped to ``1 .. p.k_top``). Move it to the device for :func:`build_mask`."""
+    out = torch.empty((n_query_blocks(p),), dtype=torch.int32)
+    stream_k_schedule(p, s, out.data_ptr())
+    return out
 
 
 def sparse_attention(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, mask: torch.Tensor, *, block_q: int,

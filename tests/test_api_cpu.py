@@ -112,3 +112,39 @@ def test_effective_k_follows_the_printed_formula(S):
     assert S.effective_k(1000, 32, 1.0) == 31          # floor(T / b_q)
     assert S.effective_k(8192, 32, 0.1) == 26           # floor(1 + 255 * 0.1)
     assert S.effective_k(64, 64, 0.5) == 1
+
+
+@pytest.mark.parametrize("kw,s", [
+    (dict(T=5000, k_top=9), 0.1), (dict(T=4096, k_top=32, causal=0), 0.3), (dict(T=777, block_q=16, block_k=16, d=64, k_top=5), 0.05),
+    (dict(T=1000, block_q=32, block_k=8, d=64, k_top=12), 0.2), (dict(T=64, k_top=3), 0.9),
+])
+def test_k_schedule_is_host_only_and_matches_the_oracle(S, kw, s):
+    """The per-row k schedule needs no GPU: checked here against the oracle's own formula."""
+    import numpy as np
+    import torch
+
+    from oracle import stream_oracle as so
+
+    p = good_problem(S, **kw)
+    got = S.k_schedule(p, s)
+    assert got.dtype == torch.int32 and not got.is_cuda
+    op = so.OracleProblem(p.batch, p.n_q_heads, p.n_kv_heads, p.T, p.d, p.block_q, p.block_k, p.k_top, bool(p.causal), "bf16")
+    np.testing.assert_array_equal(got.numpy(), so.k_schedule(op, s))
+    assert got.min() >= 1 and got.max() <= p.k_top
+
+
+def test_k_schedule_and_variable_k_reject_bad_arguments(S):
+    import torch
+
+    p = good_problem(S)
+    out = torch.zeros(4, dtype=torch.int32)
+    for s in (0.0, 1.0, -0.5, float("nan")):
+        with pytest.raises(S.StreamError) as e:
+            S.stream_k_schedule(p, s, out.data_ptr())
+        assert e.value.status == S.STREAM_ERR_INVALID_ARG
+    with pytest.raises(S.StreamError) as e:
+        S.stream_k_schedule(p, 0.5, None)
+    assert e.value.status == S.STREAM_ERR_INVALID_ARG
+    with pytest.raises(S.StreamError) as e:  # a missing schedule is an error, not the fixed-k build
+        S.stream_build_mask_var(p, 256, 256, None, 256, None, 256, 256, stream=0)
+    assert e.value.status == S.STREAM_ERR_INVALID_ARG

@@ -81,3 +81,29 @@ def test_config5_sweep(S, T):
     spec = wl.SPECS["sweep"].scaled(T=T)
     n = spec.n_rows if T <= 16384 else (1024 if T <= 262144 else 384)
     run_config(S, spec, n, n_attn_rows=32)
+
+
+def test_config3_cot_layer_128k_variable_k_sampled(S):
+    """The headline shape with k growing down the causal pattern (effective sparsity 1/128: k from
+    1 to 16 and, clamped, 16 for the lower half): a row sample against the oracle, the per-row
+    count on every row."""
+    spec = wl.SPECS["cot_layer_128k"]
+    w = wl.generate(spec)
+    q, k, _ = w.torch_tensors("cuda")
+    p = oracle_problem(spec, k_top=16)
+    k_row = so.k_schedule(p, 1.0 / 128)
+    assert k_row.min() == 1 and k_row.max() == 16
+    res = S.build_mask(q, k, block_q=spec.block, block_k=spec.block, k_top=16, k_row=torch.from_numpy(k_row).cuda())
+    torch.cuda.synchronize()
+    st = res.stats()
+    assert st.error == 0 and st.rows == spec.n_rows
+    mask = res.mask.cpu().numpy().reshape(-1, 16)
+    qb = np.arange(mask.shape[0]) % spec.n_blocks
+    assert ((mask >= 0).sum(1) == np.minimum(k_row[qb], qb + 1)).all()
+    kept = np.where(mask >= 0, mask, -1)
+    assert (np.diff(np.where(mask >= 0, mask, 1 << 30), axis=1) > 0)[mask[:, 1:] >= 0].all() and (kept.max(1) <= qb).all()
+    rows = sample_rows(spec, 2048, seed=7)
+    ora = so.build_mask_rows_var(p, w.q, w.k, k_row, rows, score_cache=True)
+    report = compare_masks(mask[rows], ora)
+    print("variable k", report, "tiles", st.tiles_scored)
+    assert report["bad"] == 0, report

@@ -328,3 +328,97 @@ def test_mask_difference_of_two_budgets(S):
     b = rng.integers(-1, 300, size=(257, 45)).astype(np.int32)
     d2, _ = S.mask_difference(torch.from_numpy(a).cuda(), torch.from_numpy(b).cuda())
     assert np.array_equal(d2.cpu().numpy(), so.mask_difference(a, b)[0])
+
+
+def variable_k_parity(S, w, k_row, *, impl, attention=True, **kw):
+    """Mask rows built with k = k_row[query block] against the oracle's (bit-exact outside ties),
+    kept scores, the tile counter, the row counts, and Eq. 2 on the oracle's variable-k mask."""
+    spec = w.spec
+    p = oracle_problem(spec, **kw)
+    bq, bk = p.block_q, p.block_k
+    q, k, v = w.torch_tensors("cuda")
+    k_dev = torch.from_numpy(k_row).cuda()
+    res = S.build_mask(q, k, block_q=bq, block_k=bk, k_top=p.k_top, causal=p.causal, impl=impl, want_scores=True, k_row=k_dev)
+    torch.cuda.synchronize()
+    st = res.stats()
+    assert st.error == 0, f"device error {st.error} (info {st.error_info:#x})"
+    mask = res.mask.cpu().numpy().reshape(-1, p.k_top)
+    ora = so.build_mask_rows_var(p, w.q, w.k, k_row, want_scores=True)
+    report = compare_masks(mask, ora)
+    assert report["bad"] == 0, report
+    same = (mask == ora["mask"]).all(axis=1)
+    sc = res.scores.cpu().numpy().reshape(-1, p.k_top)
+    fin = np.isfinite(ora["scores"][same])
+    np.testing.assert_allclose(sc[same][fin], ora["scores"][same][fin], rtol=2e-5, atol=2e-5)
+    assert (sc[same][~fin] == -np.inf).all()
+    # every row holds min(its k, blocks it may look at) entries
+    nqb = so.num_query_blocks(p)
+    qb = np.arange(mask.shape[0]) % nqb
+    last_tok = np.minimum(qb * bq + bq - 1, spec.T - 1) if p.causal else np.full(qb.shape, spec.T - 1)
+    want_cnt = np.minimum(np.clip(k_row[qb], 1, p.k_top), last_tok // bk + 1)
+    assert ((mask >= 0).sum(1) == want_cnt).all()
+    assert st.rows == mask.shape[0]
+    if same.all() and (ora["min_gap"] >= 1e-5).all():
+        assert st.tiles_scored == int(ora["tiles"].sum())
+    if attention:
+        mdev = torch.from_numpy(ora["mask"].reshape(spec.batch, spec.n_q_heads, nqb, p.k_top)).cuda()
+        out = S.sparse_attention(q, k, v, mdev, block_q=bq, block_k=bk, causal=p.causal, impl=impl)
+        torch.cuda.synchronize()
+        ref = so.sparse_attention_rows(p, w.q, w.k, w.v, ora["mask"])
+        got = out.float().cpu().numpy().reshape(-1, spec.T, spec.d)
+        for i in range(mask.shape[0]):
+            bh, b_ = divmod(i, nqb)
+            lo, hi = b_ * bq, min(spec.T, b_ * bq + bq)
+            assert np.abs(got[bh, lo:hi] - ref[i, : hi - lo]).max() <= ATTN_TOL[spec.dtype]
+    return report
+
+
+@pytest.mark.parametrize("impl", ["tensor", "generic"])
+@pytest.mark.parametrize("kw,s", [
+    (dict(T=5000, k_top=12, n_q_heads=7, n_kv_heads=1), 0.15),    # groups of 4 + 3 heads, ragged T, k from 1 to 12
+    (dict(T=8192, k_top=32, n_q_heads=4, n_kv_heads=2), 0.3),     # k reaches the row width a quarter of the way down
+    (dict(T=3000, k_top=6, n_q_heads=6, n_kv_heads=2, batch=2, local=True), 0.12),
+])
+def test_variable_k_follows_the_schedule(S, impl, kw, s):
+    w = wl.generate(tc_spec(**kw))
+    p = oracle_problem(w.spec)
+    k_row = so.k_schedule(p, s)
+    assert k_row.min() == 1 and k_row.max() == p.k_top and len(np.unique(k_row)) > 2
+    # the library's own schedule is the same one
+    sp = S.make_problem(*w.torch_tensors("cuda")[:2], block_q=64, block_k=64, k_top=p.k_top, causal=True)
+    assert np.array_equal(S.k_schedule(sp, s).numpy(), k_row)
+    variable_k_parity(S, w, k_row, impl=impl)
+
+
+@pytest.mark.parametrize("impl", ["tensor", "generic"])
+def test_variable_k_arbitrary_rows_and_clamping(S, impl):
+    """k jumps up and down from one query block to the next (levels change with it) and holds
+    entries outside 1 .. k_top, which are clamped."""
+    w = wl.generate(tc_spec(T=6000, k_top=16, n_q_heads=8, n_kv_heads=2, anchors=True))
+    nqb = -(-6000 // 64)
+    rng = np.random.default_rng(3)
+    k_row = rng.integers(1, 17, size=nqb).astype(np.int32)
+    k_row[[5, 40]] = 0
+    k_row[[6, 41]] = 99
+    k_row[-1], k_row[-2] = 1, 16
+    variable_k_parity(S, w, k_row, impl=impl)
+
+
+def test_variable_k_non_causal_and_unequal_blocks_generic(S):
+    w = wl.generate(small_spec(T=700, k_top=6))
+    for causal, bq, bk in ((False, 32, 32), (True, 16, 32), (True, 1, 16)):
+        p = oracle_problem(w.spec, block_q=bq, block_k=bk, causal=causal)
+        nqb = so.num_query_blocks(p)
+        k_row = (1 + np.arange(nqb) * 7 % 6).astype(np.int32)
+        variable_k_parity(S, w, k_row, impl="generic", block_q=bq, block_k=bk, causal=causal, attention=bq > 1)
+
+
+def test_variable_k_with_a_constant_schedule_is_the_fixed_k_build(S):
+    w = wl.generate(tc_spec(T=4096, k_top=8))
+    q, k, _ = w.torch_tensors("cuda")
+    a = S.build_mask(q, k, block_q=64, block_k=64, k_top=8, want_scores=True)
+    b = S.build_mask(q, k, block_q=64, block_k=64, k_top=8, want_scores=True,
+                     k_row=torch.full((64,), 8, dtype=torch.int32, device="cuda"))
+    torch.cuda.synchronize()
+    assert torch.equal(a.mask, b.mask) and torch.equal(a.scores, b.scores)
+    assert a.stats().tiles_scored == b.stats().tiles_scored

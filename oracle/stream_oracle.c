@@ -18,7 +18,9 @@
  *   - "top-k" orders by higher fp32 score, then lower branch index h; the survivors become the
  *     next nodes in ascending h;
  *   - k counts key blocks (row width k), not k / b_k;
- *   - the constant r of the input list is unused, as in the printed body.
+ *   - the constant r of the input list is unused, as in the printed body;
+ *   - "variable k" (named in the paper as future work, never defined): each query block runs
+ *     the unchanged algorithm with a k of its own (so_build_mask_rows_var, so_k_schedule).
  * Pins (tests, CPU only): hand-worked example, brute-force block scores on integer inputs,
  * single-level == exact top-k, count/causality/ordering invariants, full mask == dense causal
  * softmax attention (checked against a library routine), an independently structured recursive
@@ -147,9 +149,22 @@ static int index_cmp(const void *a, const void *b) {
 
 /* One query block of Algorithm 2. mask_row/score_row have k entries (ascending block index,
  * then -1 / -inf padding). Returns 0, or -1 on allocation failure. */
+static int stream_row_seen(const so_problem *p, const void *Q, const void *K, int64_t b, int64_t h, int64_t q,
+                           int n_it_override, int flags, int32_t *mask_row, float *score_row, float *min_gap,
+                           int64_t *tiles, unsigned char *seen_shared);
+
 static int stream_row(const so_problem *p, const void *Q, const void *K, int64_t b, int64_t h, int64_t q,
                       int n_it_override, int flags, int32_t *mask_row, float *score_row, float *min_gap,
                       int64_t *tiles) {
+    return stream_row_seen(p, Q, K, b, h, q, n_it_override, flags, mask_row, score_row, min_gap, tiles, NULL);
+}
+
+/* seen_shared: NULL, or N_k flags owned by the caller that say which representatives of this row
+ * were already scored by an earlier run (another k); *tiles then counts only the new ones. The
+ * scores themselves are always computed here: sharing changes the count, never a value. */
+static int stream_row_seen(const so_problem *p, const void *Q, const void *K, int64_t b, int64_t h, int64_t q,
+                           int n_it_override, int flags, int32_t *mask_row, float *score_row, float *min_gap,
+                           int64_t *tiles, unsigned char *seen_shared) {
     const int64_t k = p->k_top;
     const int64_t N_k = padded_len(p) / p->block_k;
     int n_it = 0;
@@ -161,7 +176,7 @@ static int stream_row(const so_problem *p, const void *Q, const void *K, int64_t
     float *s = malloc(sizeof(float) * 2 * k);
     ranked *order = malloc(sizeof(ranked) * 2 * k);
     int32_t *t = malloc(sizeof(int32_t) * k);
-    unsigned char *seen = calloc((size_t)N_k, 1); /* reps this row has scored */
+    unsigned char *seen = calloc((size_t)N_k, 1); /* reps this run has scored */
     unsigned char *Cblk = malloc((size_t)N_k);    /* row q of C^blk */
     float *cache = malloc(sizeof(float) * (size_t)N_k);
     if (!f || !l || !Bf || !Bl || !s || !order || !t || !seen || !cache || !Cblk) return -1;
@@ -191,7 +206,11 @@ static int stream_row(const so_problem *p, const void *Q, const void *K, int64_t
             if (!omega) { s[hh] = -INFINITY; continue; }
             int64_t r = Bf[hh];
             while (!Cblk[r]) ++r; /* first valid block of the branch */
-            if (!seen[r]) { seen[r] = 1; ++n_tiles; cache[r] = NAN; }
+            if (!seen[r]) {
+                seen[r] = 1; cache[r] = NAN;
+                if (!seen_shared) ++n_tiles;
+                else if (!seen_shared[r]) { seen_shared[r] = 1; ++n_tiles; }
+            }
             if ((flags & SO_SCORE_CACHE) && !isnan(cache[r])) s[hh] = cache[r];
             else s[hh] = cache[r] = tile_score(p, Q, K, b, h, q, r);
         }
@@ -294,6 +313,52 @@ int so_build_mask_rows_var(const so_problem *p, const void *Q, const void *K, co
             if (score_out) score_out[i * p->k_top + j] = j < pq.k_top ? sc[j] : -INFINITY;
         }
         free(m); free(sc);
+    }
+    return err;
+}
+
+/*
+ * Algorithm 2 for several sparsity constants at once (the search over k of Section 3 and the
+ * k_success / k_fail comparison of Section 4.2 need the masks of the same inputs for more than
+ * one k). Mask i is the unchanged algorithm with k = k_list[i] (1 .. k_top); a block's score
+ * does not depend on k, so an implementation may score each (row, block) tile once for all k.
+ *   mask_out  [n_k, n_rows, k_top], score_out likewise (optional), min_gap_out [n_k, n_rows]
+ *   tiles_out [n_rows]  optional: distinct representative blocks scored over ALL k of the row
+ */
+int so_build_mask_rows_multi(const so_problem *p, const void *Q, const void *K, int32_t n_k, const int32_t *k_list,
+                             const int64_t *rows, int64_t n_rows, int32_t *mask_out, float *score_out,
+                             float *min_gap_out, int64_t *tiles_out, int flags) {
+    int rc = check_problem(p);
+    if (rc) return rc;
+    if (!k_list || n_k < 1) return -2;
+    for (int32_t i = 0; i < n_k; ++i) if (k_list[i] < 1 || k_list[i] > p->k_top) return -2;
+    const int64_t Nq = so_num_query_blocks(p), total = so_num_rows(p), N_k = padded_len(p) / p->block_k;
+    int err = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t i = 0; i < n_rows; ++i) {
+        int64_t id = rows ? rows[i] : i;
+        if (id < 0 || id >= total) { err = -3; continue; }
+        int64_t q = id % Nq, h = (id / Nq) % p->n_q_heads, b = id / Nq / p->n_q_heads;
+        unsigned char *seen = calloc((size_t)N_k, 1);
+        int32_t *m = malloc(sizeof(int32_t) * p->k_top);
+        float *sc = malloc(sizeof(float) * p->k_top);
+        if (!seen || !m || !sc) { err = -1; free(seen); free(m); free(sc); continue; }
+        int64_t n_tiles = 0;
+        for (int32_t j = 0; j < n_k; ++j) {
+            so_problem pk = *p;
+            pk.k_top = k_list[j];
+            int64_t fresh = 0;
+            int64_t o = ((int64_t)j * n_rows + i);
+            if (stream_row_seen(&pk, Q, K, b, h, q, -1, flags, m, sc, min_gap_out ? min_gap_out + o : NULL, &fresh, seen))
+                err = -1;
+            n_tiles += fresh;
+            for (int64_t c = 0; c < p->k_top; ++c) {
+                mask_out[o * p->k_top + c] = c < pk.k_top ? m[c] : -1;
+                if (score_out) score_out[o * p->k_top + c] = c < pk.k_top ? sc[c] : -INFINITY;
+            }
+        }
+        if (tiles_out) tiles_out[i] = n_tiles;
+        free(seen); free(m); free(sc);
     }
     return err;
 }

@@ -104,6 +104,9 @@ def _load():
         lib.so_build_mask_rows_var.restype = ctypes.c_int
         lib.so_build_mask_rows_var.argtypes = [ctypes.POINTER(_CProblem), vp, vp, vp, i64p, ctypes.c_int64,
                                                vp, vp, vp, vp, ctypes.c_int]
+        lib.so_build_mask_rows_multi.restype = ctypes.c_int
+        lib.so_build_mask_rows_multi.argtypes = [ctypes.POINTER(_CProblem), vp, vp, ctypes.c_int32, vp, i64p,
+                                                 ctypes.c_int64, vp, vp, vp, vp, ctypes.c_int]
         lib.so_k_schedule.restype = ctypes.c_int
         lib.so_k_schedule.argtypes = [ctypes.POINTER(_CProblem), ctypes.c_double, vp]
         lib.so_sparse_attention_rows.restype = ctypes.c_int
@@ -190,6 +193,31 @@ def build_mask_rows_var(p: OracleProblem, q: np.ndarray, k: np.ndarray, k_row: n
                                     SCORE_CACHE if score_cache else 0)
     if rc:
         raise RuntimeError(f"so_build_mask_rows_var failed with {rc}")
+    out = {"mask": mask, "min_gap": gap, "tiles": tiles}
+    if want_scores:
+        out["scores"] = scores
+    return out
+
+
+def build_mask_rows_multi(p: OracleProblem, q: np.ndarray, k: np.ndarray, k_list, rows=None, *,
+                          score_cache: bool = False, want_scores: bool = False):
+    """Algorithm 2 for every k in ``k_list`` (each 1 .. k_top). Returns ``mask`` int32
+    [n_k, n, k_top], ``min_gap`` [n_k, n], ``tiles`` int64 [n] (distinct tiles over all k of a row)
+    and, if asked, ``scores`` [n_k, n, k_top]."""
+    _check(p, q, p.n_q_heads, "q"), _check(p, k, p.n_kv_heads, "k")
+    lib = _load()
+    ks = np.ascontiguousarray(k_list, dtype=np.int32)
+    rows_arr = None if rows is None else np.ascontiguousarray(rows, dtype=np.int64)
+    n = num_rows(p) if rows_arr is None else rows_arr.shape[0]
+    mask = np.empty((len(ks), n, p.k_top), np.int32)
+    gap = np.empty((len(ks), n), np.float32)
+    tiles = np.empty((n,), np.int64)
+    scores = np.empty((len(ks), n, p.k_top), np.float32) if want_scores else None
+    rc = lib.so_build_mask_rows_multi(ctypes.byref(p.c()), _ptr(q), _ptr(k), len(ks), _ptr(ks), _ptr(rows_arr), n,
+                                      _ptr(mask), _ptr(scores), _ptr(gap), _ptr(tiles),
+                                      SCORE_CACHE if score_cache else 0)
+    if rc:
+        raise RuntimeError(f"so_build_mask_rows_multi failed with {rc}")
     out = {"mask": mask, "min_gap": gap, "tiles": tiles}
     if want_scores:
         out["scores"] = scores

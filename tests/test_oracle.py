@@ -465,3 +465,38 @@ def test_k_schedule_closed_form(causal):
     assert got.max() == k_top and (not causal or got[0] == 1)  # the clamp is reached
     with pytest.raises(RuntimeError):
         so.k_schedule(p, 1.0)
+
+
+@pytest.mark.parametrize("case", [RANDOM_CASES[1], RANDOM_CASES[3], RANDOM_CASES[6], RANDOM_CASES[7]])
+def test_several_k_at_once_match_the_simulation_and_count_shared_tiles(case):
+    """Mask i of the multi-k build is Algorithm 2 with k_list[i]; the tile count of a row is the
+    size of the UNION of the representatives the simulation scores for the different k."""
+    import dataclasses
+
+    B, H, G, T, d, bq, bk, k, causal, dtype = case
+    rng = np.random.default_rng(hash(case) % (2**32) + 2)
+    q = grid_inputs(rng, (B, H, T, d), dtype, 1 / 16)
+    kk = grid_inputs(rng, (B, G, T, d), dtype, 1 / 16)
+    k_list = sorted({1, max(1, k // 2), k})
+    p = so.OracleProblem(B, H, G, T, d, bq, bk, k, causal, dtype)
+    got = so.build_mask_rows_multi(p, q, kk, k_list, want_scores=True)
+    nq_rows = so.num_query_blocks(p)
+    assert got["mask"].shape == (len(k_list), B * H * nq_rows, k)
+    shared_less = False
+    for b in range(B):
+        for h in range(H):
+            table, _, nk = block_score_table(p, q, kk, b, h)
+            for qb in range(nq_rows):
+                i = (b * H + h) * nq_rows + qb
+                union, total = set(), 0
+                for j, kj in enumerate(k_list):
+                    kept, scored, _ = simulate_row(dataclasses.replace(p, k_top=kj), table, nk, qb)
+                    assert got["mask"][j, i].tolist() == padded(kept, k), (case, b, h, qb, kj)
+                    assert got["scores"][j, i, : len(kept)].tolist() == [float(table[qb, r]) for r in kept]
+                    union |= scored
+                    total += len(scored)
+                assert got["tiles"][i] == len(union)
+                shared_less |= len(union) < total
+    assert shared_less  # the k do share representatives
+    single = so.build_mask_rows(dataclasses.replace(p, k_top=k_list[-1]), q, kk)["mask"]
+    np.testing.assert_array_equal(got["mask"][-1][:, : k_list[-1]], single)

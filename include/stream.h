@@ -127,6 +127,26 @@ stream_status stream_build_mask_var(const stream_problem *p, const void *q, cons
                                     void *cuda_stream);
 
 /*
+ * The masks of the same inputs for several sparsity constants in one call: the search over k of
+ * Section 3 (binary search for the smallest k that keeps the model's behaviour) and the
+ * k_success / k_fail comparison of Section 4.2 need them. Mask i is Algorithm 2 with
+ * k = k_list_host[i]. A block's score does not depend on k, so where the kernel can keep a row's
+ * scores (the generic kernel, while ceil(T/block_k) floats fit in shared memory beside its tiles)
+ * every (row, block) tile is scored once for all k; the tensor-core kernel is launched once per k.
+ * stream_read_stats then reports the tiles actually scored over the whole call.
+ *
+ *   n_k          1 .. 8
+ *   k_list_host  HOST int32 [n_k], each 1 .. p->k_top (p->k_top is the row width), any order
+ *   mask_out     device int32 [n_k, batch, n_q_heads, ceil(T/block_q), k_top]; mask i is one
+ *                contiguous slab, its rows -1 padded beyond k_list_host[i] entries
+ *   score_out    device float32, same shape, or NULL
+ * Everything else, and the errors, as stream_build_mask.
+ */
+stream_status stream_build_mask_multi(const stream_problem *p, const void *q, const void *k, int32_t n_k,
+                                      const int32_t *k_list_host, int32_t *mask_out, float *score_out, void *workspace,
+                                      size_t workspace_bytes, void *cuda_stream);
+
+/*
  * A schedule for stream_build_mask_var, computed on the host: the effective-sparsity formula of
  * Section 4.2, k = floor(1 + (n - 1) s), applied per query block with n = the number of key
  * blocks that row may look at (qb + 1 blocks under a causal mask with equal block sizes; the

@@ -64,6 +64,7 @@ stream_status make_geom(const stream_problem *p, Geom *g) {
     g->n_qb = (int)n_qb; g->N_k = (int)N_k;
     g->levels = levels_for((int)N_k, p->k_top);
     g->k_row = nullptr;
+    g->k_override = 0;
     g->qs_b = p->q_stride_b; g->qs_h = p->q_stride_h; g->qs_t = p->q_stride_t;
     g->ks_b = p->kv_stride_b; g->ks_h = p->kv_stride_h; g->ks_t = p->kv_stride_t;
     return STREAM_OK;
@@ -174,6 +175,57 @@ stream_status stream_build_mask_var(const stream_problem *p, const void *q, cons
                                     void *cuda_stream) {
     if (k_row == nullptr) { set_error("k_row must not be NULL (use stream_build_mask for one k)"); return STREAM_ERR_INVALID_ARG; }
     return build_mask_impl(p, q, k, k_row, mask_out, score_out, workspace, workspace_bytes, cuda_stream);
+}
+
+stream_status stream_build_mask_multi(const stream_problem *p, const void *q, const void *k, int32_t n_k,
+                                      const int32_t *k_list_host, int32_t *mask_out, float *score_out, void *workspace,
+                                      size_t workspace_bytes, void *cuda_stream) {
+    Geom g;
+    stream_status rc = make_geom(p, &g);
+    if (rc != STREAM_OK) return rc;
+    if (q == nullptr || k == nullptr || mask_out == nullptr || k_list_host == nullptr) {
+        set_error("q, k, k_list_host and mask_out must not be NULL");
+        return STREAM_ERR_INVALID_ARG;
+    }
+    if (n_k < 1 || n_k > kMaxMultiK) { set_error("between 1 and %d sparsity constants per call (got %d)", kMaxMultiK, n_k); return STREAM_ERR_INVALID_ARG; }
+    MultiK mk = {};
+    mk.n = n_k;
+    for (int i = 0; i < n_k; ++i) {
+        if (k_list_host[i] < 1 || k_list_host[i] > g.k_top) {
+            set_error("k_list_host[%d] = %d outside 1 .. k_top = %d", i, k_list_host[i], g.k_top);
+            return STREAM_ERR_INVALID_ARG;
+        }
+        mk.k[i] = k_list_host[i];
+    }
+    if (workspace == nullptr || workspace_bytes < sizeof(WorkspaceHeader) || ((uintptr_t)workspace & 255) != 0) {
+        set_error("workspace must be a 256-byte aligned device buffer of at least %zu bytes", sizeof(WorkspaceHeader));
+        return STREAM_ERR_WORKSPACE;
+    }
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    WorkspaceHeader *ws = (WorkspaceHeader *)workspace;
+    const bool tc_ok = mask_tc_supported(g, p->dtype);
+    if (p->impl == STREAM_IMPL_TENSOR && !tc_ok) {
+        set_error("tensor-core mask kernel needs bf16, d = 128, block_q = block_k = 64, k_top <= 32, 16-byte aligned strides");
+        return STREAM_ERR_UNSUPPORTED;
+    }
+    cudaError_t e = cudaMemsetAsync(ws, 0, sizeof(WorkspaceHeader), st);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(workspace)");
+    if (!(tc_ok && p->impl != STREAM_IMPL_GENERIC))
+        return launch_mask_generic_multi(g, mk, p->dtype, q, k, mask_out, score_out, ws, st);
+    // tensor-core kernel: one launch per k on the same stream (the counters add up; the work
+    // counter of the persistent kernel starts again at 0 for each)
+    const size_t per_k = (size_t)g.batch * g.H * g.n_qb * g.k_top;
+    for (int i = 0; i < n_k; ++i) {
+        if (i > 0) {
+            e = cudaMemsetAsync(&ws->work_counter, 0, sizeof(ws->work_counter), st);
+            if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(work counter)");
+        }
+        Geom gi = g;
+        gi.k_override = mk.k[i];
+        rc = launch_mask_tc(gi, q, k, mask_out + i * per_k, score_out != nullptr ? score_out + i * per_k : nullptr, ws, st);
+        if (rc != STREAM_OK) return rc;
+    }
+    return STREAM_OK;
 }
 
 stream_status stream_k_schedule(const stream_problem *p, double s, int32_t *k_row_host) {

@@ -17,6 +17,7 @@ struct Geom {
     int N_k;                    // key blocks after padding T to a multiple of lcm(bq, bk)
     int levels;                 // split levels that can change the result (with k = k_top)
     const int32_t *k_row;       // device, [n_qb]: k of each query block (clamped to 1 .. k_top), or NULL = k_top everywhere
+    int k_override;             // > 0: every row uses this k (one launch of a several-k build); rows stay k_top wide
     long long qs_b, qs_h, qs_t; // element strides
     long long ks_b, ks_h, ks_t;
 };
@@ -34,12 +35,23 @@ static_assert(sizeof(WorkspaceHeader) == 256, "workspace header is 256 bytes");
 
 constexpr int kMaxKTop = 1024;
 
+// Several sparsity constants in one call.
+constexpr int kMaxMultiK = 8;
+struct MultiK {
+    int n;               // 0: a single build (k from the geometry)
+    int k[kMaxMultiK];
+    int use_cache;       // generic kernel: N_k scores of the row fit in shared memory behind the tiles
+};
+
 void set_error(const char *fmt, ...);
 stream_status cuda_fail(cudaError_t e, const char *what);
 
 // Launchers (each validates what only it can support and returns UNSUPPORTED otherwise).
 stream_status launch_mask_generic(const Geom &g, int dtype, const void *q, const void *k, int32_t *mask,
                                   float *score, WorkspaceHeader *ws, cudaStream_t st);
+// mask / score: [mk.n][rows][k_top]; a row's tiles are scored once for all k where the cache fits.
+stream_status launch_mask_generic_multi(const Geom &g, const MultiK &mk, int dtype, const void *q, const void *k,
+                                        int32_t *mask, float *score, WorkspaceHeader *ws, cudaStream_t st);
 stream_status launch_attn_generic(const Geom &g, int dtype, const void *q, const void *k, const void *v,
                                   const int32_t *mask, float scale, void *out, cudaStream_t st);
 bool mask_tc_supported(const Geom &g, int dtype);
@@ -71,9 +83,15 @@ __host__ __device__ inline int levels_for(int N_k, int k) {
 
 // The sparsity constant of query block qb.
 __device__ __forceinline__ int row_k(const Geom &g, int qb) {
+    if (g.k_override > 0) return g.k_override;
     if (g.k_row == nullptr) return g.k_top;
     const int k = g.k_row[qb];
     return k < 1 ? 1 : (k > g.k_top ? g.k_top : k);
+}
+
+// Split levels of a row that runs with k = kq.
+__host__ __device__ inline int row_levels(const Geom &g, int kq) {
+    return kq == g.k_top ? g.levels : levels_for(g.N_k, kq);
 }
 
 // Last key block a row may look at (C^blk of Algorithm 2 in closed form), -1 if none.

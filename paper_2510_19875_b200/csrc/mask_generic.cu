@@ -64,7 +64,7 @@ __device__ float tile_score(const Geom &g, const float *Qs, float *Ks, float *re
 }
 
 template <typename T, int D>
-__global__ void __launch_bounds__(kThreads) mask_generic_kernel(Geom g, const T *__restrict__ q,
+__global__ void __launch_bounds__(kThreads) mask_generic_kernel(Geom g, MultiK mk, const T *__restrict__ q,
                                                                 const T *__restrict__ k, int32_t *__restrict__ mask,
                                                                 float *__restrict__ score, WorkspaceHeader *ws) {
     extern __shared__ float smem[];
@@ -77,6 +77,8 @@ __global__ void __launch_bounds__(kThreads) mask_generic_kernel(Geom g, const T 
     int *cand_f = node_l + g.k_top;      // [2k]
     int *cand_l = cand_f + 2 * g.k_top;  // [2k]
     int *keep = cand_l + 2 * g.k_top;    // [2k]
+    // several k: scores of this row by key block, NaN = not scored yet (a score does not depend on k)
+    float *cache = mk.use_cache ? (float *)(keep + 2 * g.k_top) : nullptr;  // [N_k]
     __shared__ float red[kThreads / 32];
     __shared__ int s_nodes, s_cands;
 
@@ -90,14 +92,21 @@ __global__ void __launch_bounds__(kThreads) mask_generic_kernel(Geom g, const T 
     const T *qp = q + b * g.qs_b + h * g.qs_h;
     const T *kp = k + b * g.ks_b + kvh * g.ks_h;
     const int q_lim = last_valid_block(g, qb);
-    const int kq = row_k(g, qb);  // this row's k (= k_top unless a schedule was given)
-    const int levels = g.k_row == nullptr ? g.levels : levels_for(g.N_k, kq);
+    const long long rows_total = (long long)g.batch * g.H * g.n_qb;
 
+    if (cache != nullptr)
+        for (int r = tid; r < g.N_k; r += kThreads) cache[r] = CUDART_NAN_F;
     for (int idx = tid; idx < kTile * D; idx += kThreads) {
         int m = idx / D, c = idx % D;
         long long tq = (long long)qb * g.bq + m;
         Qs[idx] = (m < g.bq && tq < g.T) ? to_float(qp[tq * g.qs_t + c]) : 0.f;
     }
+    unsigned tiles = 0;
+    const int n_pass = mk.n > 0 ? mk.n : 1;
+    for (int pass = 0; pass < n_pass; ++pass) {
+    const int kq = mk.n > 0 ? mk.k[pass] : row_k(g, qb);  // this pass's k (= k_top unless told otherwise)
+    const int levels = row_levels(g, kq);
+    __syncthreads();  // the previous pass is done with the node arrays
     if (tid == 0) {  // initial nodes tiling [0, N_k); keep those that hold an allowed block
         int n = 0;
         for (int j = 0; j < kq; ++j) {
@@ -109,7 +118,6 @@ __global__ void __launch_bounds__(kThreads) mask_generic_kernel(Geom g, const T 
     }
     __syncthreads();
 
-    unsigned tiles = 0;
     for (int level = 0; level < levels; ++level) {
         if (tid == 0) {
             int n = 0;
@@ -124,10 +132,17 @@ __global__ void __launch_bounds__(kThreads) mask_generic_kernel(Geom g, const T 
         const int n_cand = s_cands;
         for (int c = 0; c < n_cand; ++c) {
             if (isnan(cand_s[c])) {  // uniform: shared value
-                float s = tile_score<T, D>(g, Qs, Ks, red, kp, qb, cand_f[c]);
-                ++tiles;
+                const int r = cand_f[c];
+                float s = cache != nullptr ? cache[r] : CUDART_NAN_F;  // (uniform too)
+                if (isnan(s)) {
+                    s = tile_score<T, D>(g, Qs, Ks, red, kp, qb, r);
+                    ++tiles;
+                }
                 __syncthreads();
-                if (tid == 0) cand_s[c] = s;
+                if (tid == 0) {
+                    cand_s[c] = s;
+                    if (cache != nullptr) cache[r] = s;
+                }
             }
         }
         __syncthreads();
@@ -156,46 +171,57 @@ __global__ void __launch_bounds__(kThreads) mask_generic_kernel(Geom g, const T 
     if (score != nullptr) {  // only reachable with zero levels: scores were never needed
         for (int i = 0; i < n_nodes; ++i) {
             if (isnan(node_s[i])) {
-                float s = tile_score<T, D>(g, Qs, Ks, red, kp, qb, node_f[i]);
+                const int r = node_f[i];
+                float s = cache != nullptr ? cache[r] : CUDART_NAN_F;
+                if (isnan(s)) s = tile_score<T, D>(g, Qs, Ks, red, kp, qb, r);
                 __syncthreads();
-                if (tid == 0) node_s[i] = s;
+                if (tid == 0) {
+                    node_s[i] = s;
+                    if (cache != nullptr) cache[r] = s;
+                }
             }
         }
         __syncthreads();
     }
+    const long long o = (pass * rows_total + row) * g.k_top;
     for (int j = tid; j < g.k_top; j += kThreads) {
-        mask[row * g.k_top + j] = j < n_nodes ? node_f[j] : -1;
-        if (score != nullptr) score[row * g.k_top + j] = j < n_nodes ? node_s[j] : -CUDART_INF_F;
+        mask[o + j] = j < n_nodes ? node_f[j] : -1;
+        if (score != nullptr) score[o + j] = j < n_nodes ? node_s[j] : -CUDART_INF_F;
     }
+    }  // pass
     if (tid == 0) {
         atomicAdd(&ws->tiles_scored, (unsigned long long)tiles);
         atomicAdd(&ws->rows, 1ull);
     }
 }
 
+constexpr size_t kMaxDynamicSmem = 227 * 1024 - 1024;  // (the kernel has a few static words too)
+
 template <typename T, int D>
-stream_status launch(const Geom &g, const T *q, const T *k, int32_t *mask, float *score, WorkspaceHeader *ws,
+stream_status launch(const Geom &g, MultiK mk, const T *q, const T *k, int32_t *mask, float *score, WorkspaceHeader *ws,
                      cudaStream_t st) {
     size_t smem = sizeof(float) * (kTile * D + kTile * (D + 1) + 3 * (size_t)g.k_top) + sizeof(int) * 8 * (size_t)g.k_top;
+    mk.use_cache = mk.n > 1 && smem + sizeof(float) * (size_t)g.N_k <= kMaxDynamicSmem;
+    if (mk.use_cache) smem += sizeof(float) * (size_t)g.N_k;
     auto kern = mask_generic_kernel<T, D>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(mask_generic)");
     long long rows = (long long)g.batch * g.H * g.n_qb;
-    kern<<<(unsigned)rows, kThreads, smem, st>>>(g, q, k, mask, score, ws);
+    kern<<<(unsigned)rows, kThreads, smem, st>>>(g, mk, q, k, mask, score, ws);
     e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "mask_generic launch");
     return STREAM_OK;
 }
 
 template <typename T>
-stream_status dispatch_d(const Geom &g, const void *q, const void *k, int32_t *mask, float *score,
+stream_status dispatch_d(const Geom &g, const MultiK &mk, const void *q, const void *k, int32_t *mask, float *score,
                          WorkspaceHeader *ws, cudaStream_t st) {
     const T *qq = (const T *)q, *kk = (const T *)k;
     switch (g.d) {
-        case 16: return launch<T, 16>(g, qq, kk, mask, score, ws, st);
-        case 32: return launch<T, 32>(g, qq, kk, mask, score, ws, st);
-        case 64: return launch<T, 64>(g, qq, kk, mask, score, ws, st);
-        case 128: return launch<T, 128>(g, qq, kk, mask, score, ws, st);
+        case 16: return launch<T, 16>(g, mk, qq, kk, mask, score, ws, st);
+        case 32: return launch<T, 32>(g, mk, qq, kk, mask, score, ws, st);
+        case 64: return launch<T, 64>(g, mk, qq, kk, mask, score, ws, st);
+        case 128: return launch<T, 128>(g, mk, qq, kk, mask, score, ws, st);
     }
     set_error("generic mask kernel: head dim %d not in {16, 32, 64, 128}", g.d);
     return STREAM_ERR_UNSUPPORTED;
@@ -203,14 +229,20 @@ stream_status dispatch_d(const Geom &g, const void *q, const void *k, int32_t *m
 
 }  // namespace
 
-stream_status launch_mask_generic(const Geom &g, int dtype, const void *q, const void *k, int32_t *mask,
-                                  float *score, WorkspaceHeader *ws, cudaStream_t st) {
+stream_status launch_mask_generic_multi(const Geom &g, const MultiK &mk, int dtype, const void *q, const void *k,
+                                        int32_t *mask, float *score, WorkspaceHeader *ws, cudaStream_t st) {
     if (g.bq > kTile || g.bk > kTile) {
         set_error("generic mask kernel: block sizes up to %d (got %d, %d)", kTile, g.bq, g.bk);
         return STREAM_ERR_UNSUPPORTED;
     }
-    if (dtype == STREAM_F32) return dispatch_d<float>(g, q, k, mask, score, ws, st);
-    return dispatch_d<__nv_bfloat16>(g, q, k, mask, score, ws, st);
+    if (dtype == STREAM_F32) return dispatch_d<float>(g, mk, q, k, mask, score, ws, st);
+    return dispatch_d<__nv_bfloat16>(g, mk, q, k, mask, score, ws, st);
+}
+
+stream_status launch_mask_generic(const Geom &g, int dtype, const void *q, const void *k, int32_t *mask,
+                                  float *score, WorkspaceHeader *ws, cudaStream_t st) {
+    MultiK single = {};
+    return launch_mask_generic_multi(g, single, dtype, q, k, mask, score, ws, st);
 }
 
 }  // namespace stream

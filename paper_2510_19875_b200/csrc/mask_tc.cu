@@ -96,7 +96,6 @@ struct Params {
 // diverged lane issues TMA copies several times more slowly.
 __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUtensorMap *tk, Tail *tl, unsigned q_smem,
                               unsigned k_smem) {
-    const Geom &g = P.g;
     Ring st;
     unsigned grp_par = 0, jr_par[kR] = {0, 0, 0, 0};
     for (;;) {
@@ -152,7 +151,6 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
 // most of the time. All issuing warps walk the same unit order; each is run by all 32 lanes,
 // converged: warp-wide waits, one elected lane issues.
 __device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_smem, unsigned tmem_base, int which) {
-    const Geom &g = P.g;
     unsigned grp_par = 0, q_par = 0, jr_par[kR] = {0, 0, 0, 0};
     unsigned stage_seq = 0;   // stages so far, over the whole kernel (the same in every role)
     unsigned my_chains = 0;   // chains this warp has issued
@@ -323,7 +321,7 @@ __device__ void controller_role(const Params &P, Tail *tl, int lane) {
         const int q_lim = last_valid_block(g, qb);
         // the group's k: all its rows are the same query block
         const int kq = done ? g.k_top : row_k(g, qb);
-        const int levels = g.k_row == nullptr ? g.levels : levels_for(g.N_k, kq);
+        const int levels = row_levels(g, kq);
         // initial nodes: lane i holds node i (the same for every row of the group)
         int f0 = (int)(((long long)lane * g.N_k) / kq), l0 = (int)(((long long)(lane + 1) * g.N_k) / kq) - 1;
         const bool v0 = !done && lane < kq && f0 <= l0 && f0 <= q_lim;

@@ -76,6 +76,8 @@ def _load():
     lib.stream_build_mask.argtypes = [P, vp, vp, vp, vp, vp, sz, vp]
     lib.stream_build_mask_var.restype = ctypes.c_int
     lib.stream_build_mask_var.argtypes = [P, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.stream_build_mask_multi.restype = ctypes.c_int
+    lib.stream_build_mask_multi.argtypes = [P, vp, vp, ctypes.c_int32, vp, vp, vp, vp, sz, vp]
     lib.stream_k_schedule.restype = ctypes.c_int
     lib.stream_k_schedule.argtypes = [P, ctypes.c_double, vp]
     lib.stream_build_mask_static.restype = ctypes.c_int
@@ -142,6 +144,14 @@ def stream_build_mask_var(p: StreamProblem, q, k, k_row, mask_out, score_out, wo
     """Mask build with ``k = k_row[query block]`` (device int32 array) instead of one k."""
     _raise(_load().stream_build_mask_var(ctypes.byref(p), _addr(q), _addr(k), _addr(k_row), _addr(mask_out),
                                          _addr(score_out), _addr(workspace), workspace_bytes, _stream_handle(stream)))
+
+
+def stream_build_mask_multi(p: StreamProblem, q, k, n_k: int, k_list_host, mask_out, score_out, workspace,
+                            workspace_bytes: int, stream=None) -> None:
+    """Masks for the ``n_k`` sparsity constants in the HOST int32 array ``k_list_host``, one slab each."""
+    _raise(_load().stream_build_mask_multi(ctypes.byref(p), _addr(q), _addr(k), int(n_k), _addr(k_list_host),
+                                           _addr(mask_out), _addr(score_out), _addr(workspace), workspace_bytes,
+                                           _stream_handle(stream)))
 
 
 def stream_k_schedule(p: StreamProblem, s: float, k_row_host) -> None:
@@ -249,6 +259,21 @@ def build_mask(q: torch.Tensor, k: torch.Tensor, *, block_q: int, block_k: int, 
         if not k_row.is_cuda or k_row.dtype != torch.int32 or not k_row.is_contiguous() or tuple(k_row.shape) != (shape[2],):
             raise ValueError(f"k_row must be a contiguous int32 CUDA tensor of shape ({shape[2]},)")
         stream_build_mask_var(p, q, k, k_row, mask, scores, ws, ws.numel(), stream)
+    return MaskResult(mask, scores, ws)
+
+
+def build_masks(q: torch.Tensor, k: torch.Tensor, k_list, *, block_q: int, block_k: int, causal: bool = True,
+                impl: str = "auto", want_scores: bool = False, stream=None) -> MaskResult:
+    """Masks for every k in ``k_list`` in one call: ``mask`` is [len(k_list), B, H, rows, max(k_list)]."""
+    if not q.is_cuda or not k.is_cuda:
+        raise ValueError("q and k must be CUDA tensors (there is no CPU path)")
+    ks = torch.tensor(list(k_list), dtype=torch.int32)
+    p = make_problem(q, k, block_q=block_q, block_k=block_k, k_top=int(ks.max()), causal=causal, impl=impl)
+    shape = (len(ks), p.batch, p.n_q_heads, n_query_blocks(p), p.k_top)
+    mask = torch.empty(shape, dtype=torch.int32, device=q.device)
+    scores = torch.empty(shape, dtype=torch.float32, device=q.device) if want_scores else None
+    ws = new_workspace(p, q.device)
+    stream_build_mask_multi(p, q, k, len(ks), ks.data_ptr(), mask, scores, ws, ws.numel(), stream)
     return MaskResult(mask, scores, ws)
 
 

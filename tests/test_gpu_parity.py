@@ -422,3 +422,44 @@ def test_variable_k_with_a_constant_schedule_is_the_fixed_k_build(S):
     torch.cuda.synchronize()
     assert torch.equal(a.mask, b.mask) and torch.equal(a.scores, b.scores)
     assert a.stats().tiles_scored == b.stats().tiles_scored
+
+
+@pytest.mark.parametrize("impl,kw,k_list", [
+    ("generic", dict(T=2048, d=64, block=32, dtype="f32", n_q_heads=2, n_kv_heads=1, sink=False), [4, 2, 8]),
+    ("generic", dict(T=5000, n_q_heads=3, n_kv_heads=1), [3, 6, 12]),
+    ("tensor", dict(T=5000, n_q_heads=7, n_kv_heads=1), [3, 6, 12]),
+    ("tensor", dict(T=8192, n_q_heads=4, n_kv_heads=2, anchors=True), [32, 16, 8, 1]),
+])
+def test_several_k_in_one_call(S, impl, kw, k_list):
+    """Every slab of the several-k build against the oracle's mask for that k; the generic kernel
+    scores a (row, block) tile once for all k, which the tile counter shows."""
+    w = wl.generate(tc_spec(k_top=max(k_list), **kw))
+    spec = w.spec
+    q, k, _ = w.torch_tensors("cuda")
+    res = S.build_masks(q, k, k_list, block_q=spec.block, block_k=spec.block, impl=impl, want_scores=True)
+    torch.cuda.synchronize()
+    st = res.stats()
+    assert st.error == 0, f"device error {st.error} (info {st.error_info:#x})"
+    p = oracle_problem(spec)
+    ora = so.build_mask_rows_multi(p, w.q, w.k, k_list, want_scores=True)
+    mask = res.mask.cpu().numpy().reshape(len(k_list), -1, p.k_top)
+    sc = res.scores.cpu().numpy().reshape(mask.shape)
+    all_same = True
+    for i, ki in enumerate(k_list):
+        report = compare_masks(mask[i], {"mask": ora["mask"][i], "min_gap": ora["min_gap"][i]})
+        assert report["bad"] == 0, (ki, report)
+        assert (mask[i][:, ki:] == -1).all()
+        same = (mask[i] == ora["mask"][i]).all(axis=1)
+        all_same &= bool(same.all()) and bool((ora["min_gap"][i] >= 1e-5).all())
+        fin = np.isfinite(ora["scores"][i][same])
+        np.testing.assert_allclose(sc[i][same][fin], ora["scores"][i][same][fin], rtol=2e-5, atol=2e-5)
+        # the slab is what the single-k entry point gives
+        one = S.build_mask(q, k, block_q=spec.block, block_k=spec.block, k_top=ki, impl=impl)
+        assert torch.equal(one.mask, res.mask[i][..., :ki])
+    assert st.rows == mask.shape[1] * (len(k_list) if impl == "tensor" else 1)
+    if all_same:
+        separate = sum(int(so.build_mask_rows(oracle_problem(spec, k_top=ki), w.q, w.k)["tiles"].sum()) for ki in k_list)
+        if impl == "generic":
+            assert st.tiles_scored == int(ora["tiles"].sum()) < separate
+        else:
+            assert st.tiles_scored == separate

@@ -5,14 +5,17 @@
 // Candidate key blocks are fetched by TMA (128-byte swizzle) two at a time into a ring of
 // stages; one tcgen05.mma chain per (stage, row) computes K_pair (128 x 128) x Q_row^T (128 x 64)
 // into a 64-column TMEM slot; four epilogue warps reduce the slot to the two masked tile maxima
-// (Eq. 4 under C); a controller warp keeps each row's nodes in registers, ranks the 2k branch
+// (Eq. 4 under C) - there are two such groups of four, each serving one of every issuing warp's
+// two slots, because the fixed cost of a hand-over (wait, fences, arrive) is larger than the
+// reduction itself and one group alone is the longest stage of the pipeline; a controller warp keeps each row's nodes in registers, ranks the 2k branch
 // scores (higher score, then lower block index), compacts the survivors with ballots and
 // publishes the next level's fetch list. The first level's representatives are the same for
 // every row of a group, so one fetched stage serves all its rows; from the second level on a
 // left branch inherits its parent's score and only right branches are fetched.
 //
-// Roles (384 threads, the last two warps idle): warp 0 TMA producer, warps 1, 3, 8, 9 MMA issuers
-// (warp 1 owns TMEM), warp 2 controller, warps 4..7 epilogue (TMEM lane quarter = warp % 4). All roles walk the same fixed unit order
+// Roles (512 threads, the last two warps idle): warp 0 TMA producer, warps 1, 3, 12, 13 MMA
+// issuers (warp 1 owns TMEM), warp 2 controller, warps 4..7 and 8..11 the two epilogue groups
+// (TMEM lane quarter = warp % 4). All roles walk the same fixed unit order
 // (level 1: stage-major, row-minor; later levels: row-major), synchronised by mbarriers only.
 // Every wait is bounded: on a timeout the CTA records an error code in the workspace header,
 // raises a shared abort flag, drains its own copies and leaves.
@@ -25,8 +28,9 @@ namespace {
 
 using namespace tc;
 
-constexpr int kThreads = 384;
-constexpr int kMmaWarps = 4;   // warps 1, 3, 8, 9 issue the chains in turn
+constexpr int kThreads = 512;
+constexpr int kEpiGroups = 2;  // group g reduces the chains that land in slot g of their issuing warp
+constexpr int kMmaWarps = 4;   // warps 1, 3, 12, 13 issue the chains in turn
 constexpr int kR = 4;          // rows (query heads) per group
 constexpr int kStages = 4;     // K-pair stages
 constexpr int kSlots = 8;      // TMEM accumulator slots of 64 fp32 columns
@@ -35,7 +39,7 @@ constexpr int kHalfTile = kBlk * 128;          // 64 rows x 128 bytes (one 64-ch
 constexpr int kStageBytes = 4 * kHalfTile;     // [2 channel halves][2 tiles]
 constexpr int kQBytes = 2 * kR * kHalfTile;    // [2 channel halves][kR rows]
 constexpr int kMaxJobs = 64;
-constexpr int kListReaders = 1 + kMmaWarps + 4;  // producer warp, MMA warps, epilogue warps
+constexpr int kListReaders = 1 + kMmaWarps + 4 * kEpiGroups;  // producer warp, MMA warps, epilogue warps
 // A parity wait only means something to a thread that saw the phase before it complete, and an
 // arrival only if it cannot come a phase early. So every stage buffer and every TMEM slot
 // belongs to one issuing warp: stage s of the kernel's whole sequence goes, with all its chains,
@@ -206,7 +210,10 @@ __device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_
     }
 }
 
-__device__ void epilogue_role(const Params &P, Tail *tl, unsigned tmem_base, int wq, int lane) {
+// One epilogue group (four warps, one per TMEM lane quarter). Both groups walk every chain of
+// every list, but group `grp` only waits for and reduces those in slot `grp` of the issuing
+// warp's two: a slot's barriers are then used by one group only, which sees every phase of them.
+__device__ void epilogue_role(const Params &P, Tail *tl, unsigned tmem_base, int wq, int grp, int lane) {
     const Geom &g = P.g;
     unsigned grp_par = 0, jr_par[kR] = {0, 0, 0, 0};
     unsigned stage_seq = 0;
@@ -239,6 +246,7 @@ __device__ void epilogue_role(const Params &P, Tail *tl, unsigned tmem_base, int
                         const unsigned cnt = (chains >> (2 * owner)) & 3u;
                         const int slot = 2 * owner + (int)(cnt & 1u);
                         chains = (chains & ~(3u << (2 * owner))) | (((cnt + 1u) & 3u) << (2 * owner));
+                        if ((int)(cnt & 1u) != grp) continue;  // the other group's chain
                         if (!mbar_wait(smem_u32(&tl->tmem_full[slot]), cnt >> 1, tl, P.ws, 303)) return;
                         tc_fence_after();
                         if (blk >= 0) {
@@ -423,7 +431,7 @@ mask_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         for (int i = 0; i < kSlots; ++i) { mbar_init(smem_u32(&tl->tmem_full[i]), 1); mbar_init(smem_u32(&tl->tmem_empty[i]), 4); }
         mbar_init(smem_u32(&tl->q_full), 1);
         for (int i = 0; i <= kR; ++i) { mbar_init(smem_u32(&tl->jobs_ready[i]), 1); mbar_init(smem_u32(&tl->jobs_ack[i]), kListReaders); }
-        for (int i = 0; i < kR; ++i) mbar_init(smem_u32(&tl->scores_done[i]), 4);
+        for (int i = 0; i < kR; ++i) mbar_init(smem_u32(&tl->scores_done[i]), 4 * kEpiGroups);
         tl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_async_smem();
@@ -444,10 +452,10 @@ mask_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         controller_role(P, tl, lane);
     } else if (warp == 3) {
         mma_role(P, tl, q_smem, k_smem, tmem_base, 1);
-    } else if (warp == 8 || warp == 9) {
-        mma_role(P, tl, q_smem, k_smem, tmem_base, warp - 6);
-    } else if (warp >= 4 && warp < 8) {
-        epilogue_role(P, tl, tmem_base, warp & 3, lane);
+    } else if (warp == 12 || warp == 13) {
+        mma_role(P, tl, q_smem, k_smem, tmem_base, warp - 10);
+    } else if (warp >= 4 && warp < 12) {
+        epilogue_role(P, tl, tmem_base, warp & 3, (warp - 4) >> 2, lane);
     }
     __syncwarp();
 

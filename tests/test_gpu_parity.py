@@ -463,3 +463,32 @@ def test_several_k_in_one_call(S, impl, kw, k_list):
             assert st.tiles_scored == int(ora["tiles"].sum()) < separate
         else:
             assert st.tiles_scored == separate
+
+
+def test_mask_tensor_core_repeats_bit_for_bit(S):
+    """Many short groups per CTA with mixed group sizes (7 heads per kv head: groups of 4 and 3),
+    k changing from one query block to the next and short lists: the case in which a warp with
+    nothing to do in a list runs ahead of the others. Twenty launches must all give the oracle's
+    rows (the kernel's roles meet only on barriers, so a lost ordering shows up as a rare wrong
+    or missing row, not every time)."""
+    w = wl.generate(tc_spec(T=2500, k_top=9, n_q_heads=14, n_kv_heads=2, batch=3, local=True))
+    spec = w.spec
+    p = oracle_problem(spec)
+    nqb = so.num_query_blocks(p)
+    k_row = (1 + (np.arange(nqb) * 5) % 9).astype(np.int32)
+    ora = so.build_mask_rows_var(p, w.q, w.k, k_row)
+    ok_rows = ora["min_gap"] >= 1e-5
+    q, k, _ = w.torch_tensors("cuda")
+    k_dev = torch.from_numpy(k_row).cuda()
+    first = None
+    for it in range(20):
+        res = S.build_mask(q, k, block_q=64, block_k=64, k_top=9, impl="tensor", k_row=k_dev, want_scores=True)
+        torch.cuda.synchronize()
+        st = res.stats()
+        assert st.error == 0, f"launch {it}: device error {st.error} (info {st.error_info:#x})"
+        mask = res.mask.cpu().numpy().reshape(-1, 9)
+        assert (mask[ok_rows] == ora["mask"][ok_rows]).all(), f"launch {it}"
+        if first is None:
+            first = (mask, res.scores.cpu().numpy())
+        else:
+            assert np.array_equal(mask, first[0]) and np.array_equal(res.scores.cpu().numpy(), first[1]), f"launch {it}"

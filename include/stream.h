@@ -132,8 +132,10 @@ stream_status stream_build_mask_var(const stream_problem *p, const void *q, cons
  * k_success / k_fail comparison of Section 4.2 need them. Mask i is Algorithm 2 with
  * k = k_list_host[i]. A block's score does not depend on k, so where the kernel can keep a row's
  * scores (the generic kernel, while ceil(T/block_k) floats fit in shared memory beside its tiles)
- * every (row, block) tile is scored once for all k; the tensor-core kernel is launched once per k.
- * stream_read_stats then reports the tiles actually scored over the whole call.
+ * every (row, block) tile is scored once for all k. The tensor-core kernel does the same when the
+ * workspace has room for its score memory (stream_workspace_bytes_multi: 8 bytes per key block, row
+ * of a group and SM, i.e. O(T)); with only stream_workspace_bytes it is launched once per k and
+ * shares nothing. stream_read_stats then reports the tiles actually scored over the whole call.
  *
  *   n_k          1 .. 8
  *   k_list_host  HOST int32 [n_k], each 1 .. p->k_top (p->k_top is the row width), any order
@@ -142,6 +144,7 @@ stream_status stream_build_mask_var(const stream_problem *p, const void *q, cons
  *   score_out    device float32, same shape, or NULL
  * Everything else, and the errors, as stream_build_mask.
  */
+size_t stream_workspace_bytes_multi(const stream_problem *p, int32_t n_k);  /* 0 = invalid problem or n_k */
 stream_status stream_build_mask_multi(const stream_problem *p, const void *q, const void *k, int32_t n_k,
                                       const int32_t *k_list_host, int32_t *mask_out, float *score_out, void *workspace,
                                       size_t workspace_bytes, void *cuda_stream);

@@ -165,6 +165,15 @@ static stream_status build_mask_impl(const stream_problem *p, const void *q, con
     return launch_mask_generic(g, p->dtype, q, k, mask_out, score_out, ws, st);
 }
 
+size_t stream_workspace_bytes_multi(const stream_problem *p, int32_t n_k) {
+    Geom g;
+    if (make_geom(p, &g) != STREAM_OK) return 0;
+    if (n_k < 1 || n_k > kMaxMultiK) { set_error("between 1 and %d sparsity constants per call (got %d)", kMaxMultiK, n_k); return 0; }
+    size_t need = sizeof(WorkspaceHeader);
+    if (n_k > 1 && p->impl != STREAM_IMPL_GENERIC && mask_tc_supported(g, p->dtype)) need += mask_tc_score_memory_bytes(g);
+    return need;
+}
+
 stream_status stream_build_mask(const stream_problem *p, const void *q, const void *k, int32_t *mask_out,
                                 float *score_out, void *workspace, size_t workspace_bytes, void *cuda_stream) {
     return build_mask_impl(p, q, k, nullptr, mask_out, score_out, workspace, workspace_bytes, cuda_stream);
@@ -212,8 +221,13 @@ stream_status stream_build_mask_multi(const stream_problem *p, const void *q, co
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(workspace)");
     if (!(tc_ok && p->impl != STREAM_IMPL_GENERIC))
         return launch_mask_generic_multi(g, mk, p->dtype, q, k, mask_out, score_out, ws, st);
-    // tensor-core kernel: one launch per k on the same stream (the counters add up; the work
-    // counter of the persistent kernel starts again at 0 for each)
+    // tensor-core kernel, workspace large enough for its score memory: one launch walks every k of
+    // a group before it moves on, and scores each (row, block) tile once
+    const size_t score_bytes = mask_tc_score_memory_bytes(g);
+    if (score_bytes > 0 && workspace_bytes >= sizeof(WorkspaceHeader) + score_bytes)
+        return launch_mask_tc_multi(g, mk, q, k, mask_out, score_out, ws, (char *)workspace + sizeof(WorkspaceHeader), st);
+    // otherwise one launch per k on the same stream (the counters add up; the work counter of the
+    // persistent kernel starts again at 0 for each)
     const size_t per_k = (size_t)g.batch * g.H * g.n_qb * g.k_top;
     for (int i = 0; i < n_k; ++i) {
         if (i > 0) {

@@ -57,6 +57,11 @@ stream_status launch_attn_generic(const Geom &g, int dtype, const void *q, const
 bool mask_tc_supported(const Geom &g, int dtype);
 stream_status launch_mask_tc(const Geom &g, const void *q, const void *k, int32_t *mask, float *score,
                              WorkspaceHeader *ws, cudaStream_t st);
+// Several k in one launch (mk.n >= 1: mask / score are [mk.n][rows][k_top]); with score_memory
+// (mask_tc_score_memory_bytes(g) bytes, device) a (row, block) tile is scored once for all k.
+size_t mask_tc_score_memory_bytes(const Geom &g);
+stream_status launch_mask_tc_multi(const Geom &g, const MultiK &mk, const void *q, const void *k, int32_t *mask,
+                                   float *score, WorkspaceHeader *ws, void *score_memory, cudaStream_t st);
 bool attn_tc_supported(const Geom &g, int dtype);
 stream_status launch_attn_tc(const Geom &g, const void *q, const void *k, const void *v, const int32_t *mask,
                              float scale, void *out, cudaStream_t st);

@@ -61,6 +61,7 @@ struct Tail {
     int abort_flag;
     int grp_id, grp_b, grp_kvh, grp_qb, grp_h0, grp_R;
     int grp_levels;  // levels of this group's rows (they share the query block, hence k)
+    int grp_new_q;   // 0: another pass over the same rows (several k), the Q tiles are already there
     int n_jobs[kR + 1];
     int jobs_blk[kR + 1][kMaxJobs];
     float part[kR][kMaxJobs][2];
@@ -91,7 +92,18 @@ struct Params {
     int32_t *mask;
     float *score;
     WorkspaceHeader *ws;
+    // Several sparsity constants in one launch: a group runs the hierarchy once per k, with its Q
+    // tiles loaded once, and writes mask slab `pass`. A tile's score does not depend on k, so the
+    // controller remembers every (row, block) score of the group in `cache` (one entry per row
+    // and key block for each CTA: {group tag, score}) and only lists blocks no earlier pass scored.
+    MultiK mk;                      // n = 0: one pass with the geometry's k
+    unsigned long long *cache;      // [gridDim.x][kR][N_k], zeroed before the launch; NULL = no sharing
+    long long slab;                 // elements between two mask slabs
 };
+
+__device__ __forceinline__ unsigned long long cache_pack(unsigned tag, float s) {
+    return ((unsigned long long)tag << 32) | (unsigned long long)__float_as_uint(s);
+}
 
 // ----------------------------------------------------------------------------------------------
 // Roles
@@ -109,7 +121,7 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
         const int b = tl->grp_b, kvh = tl->grp_kvh, qb = tl->grp_qb, h0 = tl->grp_h0, R = tl->grp_R;
         const int levels = tl->grp_levels;
         // Q tiles of the group's rows (previous group's MMAs are all complete by now)
-        if (elect_one()) {
+        if (tl->grp_new_q && elect_one()) {
             mbar_arrive_expect_tx(smem_u32(&tl->q_full), (unsigned)(R * 2 * kHalfTile));
             for (int r = 0; r < R; ++r)
                 for (int c = 0; c < 2; ++c)
@@ -164,8 +176,10 @@ __device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_
         grp_par ^= 1;
         if (tl->grp_id < 0) return;
         const int R = tl->grp_R, levels = tl->grp_levels;
-        if (!mbar_wait_w(smem_u32(&tl->q_full), q_par, tl, P.ws, 202)) return;
-        q_par ^= 1;
+        if (tl->grp_new_q) {
+            if (!mbar_wait_w(smem_u32(&tl->q_full), q_par, tl, P.ws, 202)) return;
+            q_par ^= 1;
+        }
         for (int level = 0; level < levels; ++level) {
             const int lists = level == 0 ? 1 : R;
             for (int x = 0; x < lists; ++x) {
@@ -306,11 +320,16 @@ __device__ __forceinline__ Keep select_topk(bool vl, float sl, bool vr, float sr
     return {vl && rank_l < k, vr && rank_r < k};
 }
 
+// kMulti: several k per group with the score memory; false compiles the plain single-pass
+// controller (its ranking step is on every group's critical path, so it carries nothing extra).
+template <bool kMulti>
 __device__ void controller_role(const Params &P, Tail *tl, int lane) {
     const Geom &g = P.g;
     const unsigned lt = (1u << lane) - 1u;
     unsigned sd_par[kR] = {0, 0, 0, 0};
     unsigned ack_par[kR + 1] = {0, 0, 0, 0, 0};  // phase of the next acknowledgement of each list
+    // this CTA's score memory for the rows of its current group (several k only)
+    unsigned long long *const cache = kMulti ? P.cache + (size_t)blockIdx.x * kR * g.N_k : nullptr;
     for (;;) {
         int id = 0;
         if (lane == 0) id = (int)atomicAdd(&P.ws->work_counter, 1u);
@@ -327,97 +346,137 @@ __device__ void controller_role(const Params &P, Tail *tl, int lane) {
             R = min(kR, g.hpg - chunk * kR);
         }
         const int q_lim = last_valid_block(g, qb);
-        // the group's k: all its rows are the same query block
-        const int kq = done ? g.k_top : row_k(g, qb);
-        const int levels = row_levels(g, kq);
-        // initial nodes: lane i holds node i (the same for every row of the group)
-        int f0 = (int)(((long long)lane * g.N_k) / kq), l0 = (int)(((long long)(lane + 1) * g.N_k) / kq) - 1;
-        const bool v0 = !done && lane < kq && f0 <= l0 && f0 <= q_lim;
-        const int m0 = (f0 + l0) / 2;
-        const bool vl1 = v0, vr1 = v0 && m0 + 1 <= l0 && m0 + 1 <= q_lim;
-        const unsigned bl = __ballot_sync(0xffffffffu, vl1), br = __ballot_sync(0xffffffffu, vr1);
-        const int c_l1 = __popc(bl & lt) + __popc(br & lt), c_r1 = c_l1 + (vl1 ? 1 : 0);
-        // the previous group's first list and record have been read by everybody (passes at once the first time)
-        if (!mbar_wait(smem_u32(&tl->jobs_ack[kR]), ack_par[kR] ^ 1, tl, P.ws, 402)) return;
-        ack_par[kR] ^= 1;
-        if (vl1) tl->jobs_blk[kR][c_l1] = f0;
-        if (vr1) tl->jobs_blk[kR][c_r1] = m0 + 1;
-        const int n1 = __popc(bl) + __popc(br);
-        if (lane == 0) {
-            tl->n_jobs[kR] = n1;
-            tl->grp_id = done ? -1 : id; tl->grp_b = b; tl->grp_kvh = kvh; tl->grp_qb = qb; tl->grp_h0 = h0; tl->grp_R = R;
-            tl->grp_levels = levels;
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&tl->jobs_ready[kR]));
-        if (done) return;
-
-        int nf[kR], nl[kR], my_c[kR], n_nodes[kR];
-        float ns[kR];
-        bool has_r[kR];
-        unsigned tiles = (unsigned)(n1 * R);
-        for (int level = 0; level < levels; ++level) {
+        const unsigned tag = (unsigned)id + 1u;  // marks this group's entries of the score memory (0 = never written)
+        const int n_pass = (!kMulti || done) ? 1 : P.mk.n;
+        for (int pass = 0; pass < n_pass; ++pass) {
+            // the group's k: all its rows are the same query block
+            const int kq = done ? g.k_top : (kMulti ? P.mk.k[pass] : row_k(g, qb));
+            const int levels = row_levels(g, kq);
+            // initial nodes: lane i holds node i (the same for every row of the group)
+            int f0 = (int)(((long long)lane * g.N_k) / kq), l0 = (int)(((long long)(lane + 1) * g.N_k) / kq) - 1;
+            const bool v0 = !done && lane < kq && f0 <= l0 && f0 <= q_lim;
+            const int m0 = (f0 + l0) / 2;
+            const bool vl1 = v0, vr1 = v0 && m0 + 1 <= l0 && m0 + 1 <= q_lim;
+            // Which of the two candidates does some row still lack a score for? (Without a score
+            // memory: all of them.) A block on the first level's list is scored for every row.
+            unsigned miss_l = vl1 ? (1u << R) - 1u : 0u, miss_r = vr1 ? (1u << R) - 1u : 0u;  // bit r: row r lacks it
+            float cl[kR], cr[kR];
+            if (kMulti && !done) {
 #pragma unroll
-            for (int r = 0; r < kR; ++r) {
-                if (r >= R) continue;
-                if (!mbar_wait(smem_u32(&tl->scores_done[r]), sd_par[r], tl, P.ws, 401)) return;
-                sd_par[r] ^= 1;
-                // candidates of this lane's node: left (f : m) and right (m + 1 : l)
-                int f, l, m;
-                bool vl, vr;
-                float sl, sr = -CUDART_INF_F;
-                if (level == 0) {
-                    f = f0; l = l0; m = m0; vl = vl1; vr = vr1;
-                    sl = vl ? fmaxf(tl->part[r][c_l1][0], tl->part[r][c_l1][1]) : -CUDART_INF_F;
-                    if (vr) sr = fmaxf(tl->part[r][c_r1][0], tl->part[r][c_r1][1]);
-                } else {
-                    f = nf[r]; l = nl[r]; m = (f + l) / 2;
-                    vl = lane < n_nodes[r]; vr = has_r[r];
-                    sl = ns[r];
-                    if (vr) sr = fmaxf(tl->part[r][my_c[r]][0], tl->part[r][my_c[r]][1]);
-                }
-                const Keep kp = select_topk(vl, sl, vr, sr, kq, lane);
-                const unsigned kl = __ballot_sync(0xffffffffu, kp.l), kr = __ballot_sync(0xffffffffu, kp.r);
-                const int pos_l = __popc(kl & lt) + __popc(kr & lt), pos_r = pos_l + (kp.l ? 1 : 0);
-                __syncwarp();
-                if (kp.l) { tl->node_f[pos_l] = f; tl->node_l[pos_l] = m; tl->node_s[pos_l] = sl; }
-                if (kp.r) { tl->node_f[pos_r] = m + 1; tl->node_l[pos_r] = l; tl->node_s[pos_r] = sr; }
-                __syncwarp();
-                n_nodes[r] = __popc(kl) + __popc(kr);
-                const bool live = lane < n_nodes[r];
-                nf[r] = live ? tl->node_f[lane] : 0;
-                nl[r] = live ? tl->node_l[lane] : -1;
-                ns[r] = live ? tl->node_s[lane] : -CUDART_INF_F;
-                if (level + 1 < levels) {
-                    // next level: only right branches need a tile; left ones keep the node's score
-                    const int mm = (nf[r] + nl[r]) / 2;
-                    has_r[r] = live && nl[r] > nf[r] && mm + 1 <= q_lim;
-                    const unsigned hb = __ballot_sync(0xffffffffu, has_r[r]);
-                    my_c[r] = __popc(hb & lt);
-                    if (!mbar_wait(smem_u32(&tl->jobs_ack[r]), ack_par[r] ^ 1, tl, P.ws, 403)) return;
-                    ack_par[r] ^= 1;
-                    if (has_r[r]) tl->jobs_blk[r][my_c[r]] = mm + 1;
-                    if (lane == 0) tl->n_jobs[r] = __popc(hb);
-                    tiles += (unsigned)__popc(hb);
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&tl->jobs_ready[r]));
-                } else {
-                    // emit I[q, :]: first block of every surviving node, ascending, -1 padded
-                    const long long row = ((long long)b * g.H + (h0 + r)) * g.n_qb + qb;
-                    if (lane < g.k_top) {
-                        P.mask[row * g.k_top + lane] = live ? nf[r] : -1;
-                        if (P.score != nullptr) P.score[row * g.k_top + lane] = live ? ns[r] : -CUDART_INF_F;
+                for (int r = 0; r < kR; ++r) {
+                    cl[r] = cr[r] = -CUDART_INF_F;
+                    if (r >= R) continue;
+                    if (vl1) {
+                        const unsigned long long e = __ldcg(cache + (size_t)r * g.N_k + f0);
+                        if ((unsigned)(e >> 32) == tag) { cl[r] = __uint_as_float((unsigned)e); miss_l &= ~(1u << r); }
+                    }
+                    if (vr1) {
+                        const unsigned long long e = __ldcg(cache + (size_t)r * g.N_k + m0 + 1);
+                        if ((unsigned)(e >> 32) == tag) { cr[r] = __uint_as_float((unsigned)e); miss_r &= ~(1u << r); }
                     }
                 }
             }
-        }
-        if (lane == 0) {
-            atomicAdd(&P.ws->tiles_scored, (unsigned long long)tiles);
-            atomicAdd(&P.ws->rows, (unsigned long long)R);
+            const bool fl1 = miss_l != 0u, fr1 = miss_r != 0u;  // goes on the list
+            const unsigned bl = __ballot_sync(0xffffffffu, fl1), br = __ballot_sync(0xffffffffu, fr1);
+            const int c_l1 = __popc(bl & lt) + __popc(br & lt), c_r1 = c_l1 + (fl1 ? 1 : 0);
+            // the previous list and record have been read by everybody (passes at once the first time)
+            if (!mbar_wait(smem_u32(&tl->jobs_ack[kR]), ack_par[kR] ^ 1, tl, P.ws, 402)) return;
+            ack_par[kR] ^= 1;
+            if (fl1) tl->jobs_blk[kR][c_l1] = f0;
+            if (fr1) tl->jobs_blk[kR][c_r1] = m0 + 1;
+            const int n1 = __popc(bl) + __popc(br);
+            if (lane == 0) {
+                tl->n_jobs[kR] = n1;
+                tl->grp_id = done ? -1 : id; tl->grp_b = b; tl->grp_kvh = kvh; tl->grp_qb = qb; tl->grp_h0 = h0; tl->grp_R = R;
+                tl->grp_levels = levels;
+                tl->grp_new_q = pass == 0;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&tl->jobs_ready[kR]));
+            if (done) return;
+
+            int nf[kR], nl[kR], my_c[kR], n_nodes[kR], rb[kR];
+            float ns[kR], cs[kR];
+            bool has_r[kR], need[kR];
+            unsigned tiles = 0;  // (row, block) tiles that had no score yet
+#pragma unroll
+            for (int r = 0; r < kR; ++r)
+                if (r < R) tiles += (unsigned)(__popc(__ballot_sync(0xffffffffu, (miss_l >> r) & 1u)) + __popc(__ballot_sync(0xffffffffu, (miss_r >> r) & 1u)));
+            for (int level = 0; level < levels; ++level) {
+#pragma unroll
+                for (int r = 0; r < kR; ++r) {
+                    if (r >= R) continue;
+                    if (!mbar_wait(smem_u32(&tl->scores_done[r]), sd_par[r], tl, P.ws, 401)) return;
+                    sd_par[r] ^= 1;
+                    // candidates of this lane's node: left (f : m) and right (m + 1 : l)
+                    int f, l, m;
+                    bool vl, vr;
+                    float sl = -CUDART_INF_F, sr = -CUDART_INF_F;
+                    if (level == 0) {
+                        f = f0; l = l0; m = m0; vl = vl1; vr = vr1;
+                        if (vl) sl = fl1 ? fmaxf(tl->part[r][c_l1][0], tl->part[r][c_l1][1]) : cl[r];
+                        if (vr) sr = fr1 ? fmaxf(tl->part[r][c_r1][0], tl->part[r][c_r1][1]) : cr[r];
+                        if (kMulti) {
+                            if (fl1) __stcg(cache + (size_t)r * g.N_k + f0, cache_pack(tag, sl));
+                            if (fr1) __stcg(cache + (size_t)r * g.N_k + m0 + 1, cache_pack(tag, sr));
+                        }
+                    } else {
+                        f = nf[r]; l = nl[r]; m = (f + l) / 2;
+                        vl = lane < n_nodes[r]; vr = has_r[r];
+                        sl = ns[r];
+                        if (vr) sr = need[r] ? fmaxf(tl->part[r][my_c[r]][0], tl->part[r][my_c[r]][1]) : cs[r];
+                        if (kMulti && need[r]) __stcg(cache + (size_t)r * g.N_k + rb[r], cache_pack(tag, sr));
+                    }
+                    const Keep kp = select_topk(vl, sl, vr, sr, kq, lane);
+                    const unsigned kl = __ballot_sync(0xffffffffu, kp.l), kr = __ballot_sync(0xffffffffu, kp.r);
+                    const int pos_l = __popc(kl & lt) + __popc(kr & lt), pos_r = pos_l + (kp.l ? 1 : 0);
+                    __syncwarp();
+                    if (kp.l) { tl->node_f[pos_l] = f; tl->node_l[pos_l] = m; tl->node_s[pos_l] = sl; }
+                    if (kp.r) { tl->node_f[pos_r] = m + 1; tl->node_l[pos_r] = l; tl->node_s[pos_r] = sr; }
+                    __syncwarp();
+                    n_nodes[r] = __popc(kl) + __popc(kr);
+                    const bool live = lane < n_nodes[r];
+                    nf[r] = live ? tl->node_f[lane] : 0;
+                    nl[r] = live ? tl->node_l[lane] : -1;
+                    ns[r] = live ? tl->node_s[lane] : -CUDART_INF_F;
+                    if (level + 1 < levels) {
+                        // next level: only right branches need a tile; left ones keep the node's score
+                        const int mm = (nf[r] + nl[r]) / 2;
+                        has_r[r] = live && nl[r] > nf[r] && mm + 1 <= q_lim;
+                        rb[r] = mm + 1;
+                        need[r] = has_r[r];
+                        if (kMulti && has_r[r]) {  // an earlier pass (another k) may have scored it
+                            const unsigned long long e = __ldcg(cache + (size_t)r * g.N_k + rb[r]);
+                            if ((unsigned)(e >> 32) == tag) { cs[r] = __uint_as_float((unsigned)e); need[r] = false; }
+                        }
+                        const unsigned hb = __ballot_sync(0xffffffffu, need[r]);
+                        my_c[r] = __popc(hb & lt);
+                        if (!mbar_wait(smem_u32(&tl->jobs_ack[r]), ack_par[r] ^ 1, tl, P.ws, 403)) return;
+                        ack_par[r] ^= 1;
+                        if (need[r]) tl->jobs_blk[r][my_c[r]] = rb[r];
+                        if (lane == 0) tl->n_jobs[r] = __popc(hb);
+                        tiles += (unsigned)__popc(hb);
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&tl->jobs_ready[r]));
+                    } else {
+                        // emit I[q, :]: first block of every surviving node, ascending, -1 padded
+                        const long long o = (long long)pass * P.slab + (((long long)b * g.H + (h0 + r)) * g.n_qb + qb) * g.k_top;
+                        if (lane < g.k_top) {
+                            P.mask[o + lane] = live ? nf[r] : -1;
+                            if (P.score != nullptr) P.score[o + lane] = live ? ns[r] : -CUDART_INF_F;
+                        }
+                    }
+                }
+            }
+            if (lane == 0) {
+                atomicAdd(&P.ws->tiles_scored, (unsigned long long)tiles);
+                atomicAdd(&P.ws->rows, (unsigned long long)R);
+            }
         }
     }
 }
 
+template <bool kMulti>
 __global__ void __launch_bounds__(kThreads, 1)
 mask_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k, Params P) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
@@ -449,7 +508,7 @@ mask_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     } else if (warp == 1) {
         mma_role(P, tl, q_smem, k_smem, tmem_base, 0);
     } else if (warp == 2) {
-        controller_role(P, tl, lane);
+        controller_role<kMulti>(P, tl, lane);
     } else if (warp == 3) {
         mma_role(P, tl, q_smem, k_smem, tmem_base, 1);
     } else if (warp == 12 || warp == 13) {
@@ -483,8 +542,32 @@ bool mask_tc_supported(const Geom &g, int dtype) {
            tma_strides_ok(g);
 }
 
+namespace {
+// CTAs of a launch and the groups they share.
+stream_status launch_shape(const Geom &g, int *grid, long long *n_groups) {
+    const int n_sm = sm_count();
+    if (n_sm <= 0) { set_error("cannot read the SM count of the current device"); return STREAM_ERR_CUDA; }
+    *n_groups = (long long)g.batch * g.G * g.n_qb * ((g.hpg + kR - 1) / kR);
+    *grid = (int)(*n_groups < n_sm ? *n_groups : n_sm);
+    return STREAM_OK;
+}
+}  // namespace
+
+size_t mask_tc_score_memory_bytes(const Geom &g) {
+    int grid = 0;
+    long long n_groups = 0;
+    if (launch_shape(g, &grid, &n_groups) != STREAM_OK) return 0;
+    return (size_t)grid * kR * (size_t)g.N_k * sizeof(unsigned long long);
+}
+
 stream_status launch_mask_tc(const Geom &g, const void *q, const void *k, int32_t *mask, float *score,
                              WorkspaceHeader *ws, cudaStream_t st) {
+    MultiK single = {};
+    return launch_mask_tc_multi(g, single, q, k, mask, score, ws, nullptr, st);
+}
+
+stream_status launch_mask_tc_multi(const Geom &g, const MultiK &mk, const void *q, const void *k, int32_t *mask,
+                                   float *score, WorkspaceHeader *ws, void *score_memory, cudaStream_t st) {
     if (((uintptr_t)q & 15) != 0 || ((uintptr_t)k & 15) != 0) {
         set_error("tensor-core mask kernel needs 16-byte aligned q and k");
         return STREAM_ERR_UNSUPPORTED;
@@ -500,12 +583,22 @@ stream_status launch_mask_tc(const Geom &g, const void *q, const void *k, int32_
     long long n_groups = (long long)g.batch * g.G * g.n_qb * P.n_chunks;
     P.n_groups = (int)n_groups;
     P.mask = mask; P.score = score; P.ws = ws;
-    const int n_sm = sm_count();
-    if (n_sm <= 0) { set_error("cannot read the SM count of the current device"); return STREAM_ERR_CUDA; }
-    cudaError_t e = cudaFuncSetAttribute(mask_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    P.mk = mk;
+    P.cache = (unsigned long long *)score_memory;
+    P.slab = (long long)g.batch * g.H * g.n_qb * g.k_top;
+    int grid = 0;
+    rc = launch_shape(g, &grid, &n_groups);
+    if (rc != STREAM_OK) return rc;
+    cudaError_t e = cudaSuccess;
+    if (score_memory != nullptr) {  // tag 0 = "no score yet"
+        e = cudaMemsetAsync(score_memory, 0, mask_tc_score_memory_bytes(g), st);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(score memory)");
+    }
+    if (mk.n >= 1 && score_memory == nullptr) { set_error("several k in one launch need the score memory"); return STREAM_ERR_WORKSPACE; }
+    auto kern = mk.n >= 1 ? mask_tc_kernel<true> : mask_tc_kernel<false>;
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(mask_tc)");
-    int grid = (int)(n_groups < n_sm ? n_groups : n_sm);
-    mask_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(tq, tk, P);
+    kern<<<grid, kThreads, kSmemBytes, st>>>(tq, tk, P);
     e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "mask_tc launch");
     return STREAM_OK;

@@ -76,6 +76,8 @@ def _load():
     lib.stream_build_mask.argtypes = [P, vp, vp, vp, vp, vp, sz, vp]
     lib.stream_build_mask_var.restype = ctypes.c_int
     lib.stream_build_mask_var.argtypes = [P, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.stream_workspace_bytes_multi.restype = sz
+    lib.stream_workspace_bytes_multi.argtypes = [P, ctypes.c_int32]
     lib.stream_build_mask_multi.restype = ctypes.c_int
     lib.stream_build_mask_multi.argtypes = [P, vp, vp, ctypes.c_int32, vp, vp, vp, vp, sz, vp]
     lib.stream_k_schedule.restype = ctypes.c_int
@@ -144,6 +146,11 @@ def stream_build_mask_var(p: StreamProblem, q, k, k_row, mask_out, score_out, wo
     """Mask build with ``k = k_row[query block]`` (device int32 array) instead of one k."""
     _raise(_load().stream_build_mask_var(ctypes.byref(p), _addr(q), _addr(k), _addr(k_row), _addr(mask_out),
                                          _addr(score_out), _addr(workspace), workspace_bytes, _stream_handle(stream)))
+
+
+def stream_workspace_bytes_multi(p: StreamProblem, n_k: int) -> int:
+    """Workspace with which a several-k build scores every (row, block) tile once (0 = invalid)."""
+    return int(_load().stream_workspace_bytes_multi(ctypes.byref(p), int(n_k)))
 
 
 def stream_build_mask_multi(p: StreamProblem, q, k, n_k: int, k_list_host, mask_out, score_out, workspace,
@@ -263,8 +270,10 @@ def build_mask(q: torch.Tensor, k: torch.Tensor, *, block_q: int, block_k: int, 
 
 
 def build_masks(q: torch.Tensor, k: torch.Tensor, k_list, *, block_q: int, block_k: int, causal: bool = True,
-                impl: str = "auto", want_scores: bool = False, stream=None) -> MaskResult:
-    """Masks for every k in ``k_list`` in one call: ``mask`` is [len(k_list), B, H, rows, max(k_list)]."""
+                impl: str = "auto", want_scores: bool = False, share: bool = True, stream=None) -> MaskResult:
+    """Masks for every k in ``k_list`` in one call: ``mask`` is [len(k_list), B, H, rows, max(k_list)].
+    ``share=False`` gives the library only the small workspace (the tensor-core kernel then runs
+    once per k and does not reuse tile scores between them)."""
     if not q.is_cuda or not k.is_cuda:
         raise ValueError("q and k must be CUDA tensors (there is no CPU path)")
     ks = torch.tensor(list(k_list), dtype=torch.int32)
@@ -272,7 +281,10 @@ def build_masks(q: torch.Tensor, k: torch.Tensor, k_list, *, block_q: int, block
     shape = (len(ks), p.batch, p.n_q_heads, n_query_blocks(p), p.k_top)
     mask = torch.empty(shape, dtype=torch.int32, device=q.device)
     scores = torch.empty(shape, dtype=torch.float32, device=q.device) if want_scores else None
-    ws = new_workspace(p, q.device)
+    n_ws = stream_workspace_bytes_multi(p, len(ks)) if share else stream_workspace_bytes(p)
+    if n_ws == 0:
+        raise StreamError(STREAM_ERR_INVALID_ARG, stream_last_error())
+    ws = torch.empty(n_ws, dtype=torch.uint8, device=q.device)
     stream_build_mask_multi(p, q, k, len(ks), ks.data_ptr(), mask, scores, ws, ws.numel(), stream)
     return MaskResult(mask, scores, ws)
 

@@ -44,6 +44,7 @@ def parse_args():
     ap.add_argument("--kernels", default="auto", choices=["auto", "generic", "tensor"], help="library kernel choice")
     ap.add_argument("--k-sparsity", type=float, default=0.0,
                     help="build the mask with k per query block from this effective sparsity (0 = one k; implies --no-e2e)")
+    ap.add_argument("--k-list", default="", help="comma-separated k values: time the several-k mask build (one JSON line, masks only)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="target CPU time of the oracle sample")
@@ -471,8 +472,41 @@ def run_sweep(args):
                       "fit_peak_memory_vs_T": {"bytes_per_token": m_a, "offset_bytes": m_b, "r2": r2_mem}}))
 
 
+def run_k_list(args):
+    """The several-k mask build (the search over k of Section 3 wants the masks of one input for
+    more than one k): one call that shares tile scores between the k, against the same call with
+    the small workspace (one launch per k, nothing shared)."""
+    import torch
+
+    from paper_2510_19875_b200 import stream as S
+    from paper_2510_19875_b200 import workloads as wl
+
+    ks = [int(x) for x in args.k_list.split(",")]
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    spec = get_spec(args, 0)
+    w = wl.generate(spec)
+    q, k, _ = w.torch_tensors(dev)
+    out = {"workload": spec.name, "T": spec.T, "k_list": ks, "kernels": args.kernels}
+    for name, share in (("shared", True), ("per_k", False)):
+        best, res = float("inf"), None
+        for it in range(args.warmup + args.steps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            res = S.build_masks(q, k, ks, block_q=spec.block, block_k=spec.block, impl=args.kernels, share=share)
+            b.record()
+            torch.cuda.synchronize()
+            if it >= args.warmup:
+                best = min(best, a.elapsed_time(b))
+        out[name] = {"ms": best, "tiles_scored": int(res.stats().tiles_scored), "workspace_bytes": int(res.workspace.numel())}
+    print(json.dumps(out))
+
+
 def main():
     args = parse_args()
+    if args.k_list:
+        run_k_list(args)
+        return
     if args.sweep:
         run_sweep(args)
     elif args.impl == "reference":

@@ -50,7 +50,10 @@ constexpr int kHalfTile = kBlk * 128;       // 64 rows x 128 bytes
 constexpr int kTile = 2 * kHalfTile;        // one 64 x 128 tile
 constexpr int kOperand = 2 * kTile;         // two tiles (K_a, K_b or V_a, V_b), or the 128-row Q operand
 constexpr int kPBytes = 2 * kHalfTile;      // one group's P: 128 rows x 64 keys
-constexpr int kMaxKStages = 3, kVStages = 2;  // K stages: what shared memory allows (2 or 3); V stages = groups
+// Stages of the two rings, out of the five operand buffers shared memory has room for beside Q
+// and P (four when the mask rows are long): a V stage is held from its load until the product of
+// its entry is complete, a whole softmax later, so V gets three when there are five, K two.
+constexpr int kMaxKStages = 3, kMaxVStages = 3;
 constexpr int kMaskSlots = 2;               // pairs whose mask rows are resident
 constexpr int kMaxKTopTc = 1024;
 constexpr float kLazyLog2 = 8.f;            // ref is raised when the maximum exceeds it by this much (log2 units)
@@ -58,10 +61,9 @@ constexpr float kLazyLog2 = 8.f;            // ref is raised when the maximum ex
 // TMEM columns: S of group g at 128 g, O of group g at 256 + 128 g.
 struct Tail {
     unsigned long long q_full, q_empty;
-    unsigned long long k_full[kMaxKStages], k_empty[kMaxKStages], v_full[kVStages];
+    unsigned long long k_full[kMaxKStages], k_empty[kMaxKStages], v_full[kMaxVStages], v_empty[kMaxVStages];
     // Per group g (entries n with n % 2 == g): logits ready / read, P published, product added.
-    // o_full[g] also tells the producer that V stage g is free and the group that its P buffer
-    // is: the ring of V stages and the groups move together.
+    // o_full[g] also tells the group that its P buffer is free again.
     unsigned long long s_full[2], s_empty[2], p_full[2], o_full[2];
     unsigned long long m_full[kMaskSlots], m_empty[kMaskSlots];
     unsigned long long x_bar[4];  // the two softmax warps of a lane quarter (one per group) meet here
@@ -70,7 +72,7 @@ struct Tail {
 };
 // Dynamic shared memory: Q | P of group 0, P of group 1 | V stages | K stages | Tail | mask rows
 // [kMaskSlots][2][row_stride] (-1 where a row has nothing), the operands 1024-byte aligned.
-constexpr int kFixedOperands = 2 + kVStages;  // Q, the two P together, the V stages
+constexpr int kFixedOperands = 2;  // Q, the two P together; behind them the V stages, then the K stages
 constexpr int kMaxSmemPerCta = 232448;
 
 constexpr unsigned kIdescQK = idesc_bf16(128, 128, false);  // B = stacked K tiles, K-major
@@ -82,7 +84,7 @@ struct Params {
     int n_items, n_pairs;  // pairs per kv head: ceil(hpg / 2)
     int row_stride;        // ints per resident mask row (k_top rounded up to a multiple of 4)
     int smem_bytes;        // dynamic shared memory of the launch
-    int n_k_stages;        // set by the kernel from what fits behind its aligned base
+    int n_k_stages, n_v_stages;  // set by the kernel from what fits behind its aligned base
     const int32_t *mask;
     __nv_bfloat16 *out;
     float scale_log2;      // logit scale times log2(e)
@@ -258,10 +260,10 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
             return true;
         }
         // a V stage is free once the product computed from it is complete
-        if (!probe_w(smem_u32(&tl->o_full[S.ring.idx]), S.ring.phase ^ 1)) return false;
+        if (!probe_w(smem_u32(&tl->v_empty[S.ring.idx]), S.ring.phase ^ 1)) return false;
         if (elect_one()) load_v_pair(v_smem + S.ring.idx * kOperand, smem_u32(&tl->v_full[S.ring.idx]), S.it, S.cur);
         __syncwarp();
-        S.ring.advance(kVStages);
+        S.ring.advance(P.n_v_stages);
         S.e = next_entry(rows, P.row_stride, S.e, g.k_top, &S.cur);
         return true;
     };
@@ -334,7 +336,7 @@ __device__ void qk_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_s
 // O_g (+)= P_g [V_a; V_b] for every kept entry; a group's first entry of a pair starts its O afresh.
 __device__ void pv_role(const Params &P, Tail *tl, unsigned p_smem, unsigned v_smem, unsigned tmem_base) {
     const Geom &g = P.g;
-    Ring gr, ms;  // gr: group = V stage = O buffer of the entry
+    Ring gr, vs, ms;  // gr: group = O buffer of the entry; vs: its V stage
     // the MN-major V tiles have their two 64-channel halves kHalfTile apart
     const unsigned p_lo = desc_lo_sw128(p_smem, 16), v_lo = desc_lo_sw128(v_smem, kHalfTile);
     for (int id = blockIdx.x; id < P.n_items; id += gridDim.x) {
@@ -343,11 +345,11 @@ __device__ void pv_role(const Params &P, Tail *tl, unsigned p_smem, unsigned v_s
         const int n_entries = count_entries(rows, P.row_stride, g.k_top);
         unsigned fresh = 3u;  // bit g: group g has not added anything for this pair yet
         for (int i = 0; i < n_entries; ++i) {
-            if (!wait_w(smem_u32(&tl->v_full[gr.idx]), gr.phase, tl, 205)) return;
+            if (!wait_w(smem_u32(&tl->v_full[vs.idx]), vs.phase, tl, 205)) return;
             if (!wait_w(smem_u32(&tl->p_full[gr.idx]), gr.phase, tl, 204)) return;  // also: O_g rescaled if it had to be
             tc_fence_after();
             const unsigned d_tmem = tmem_base + 256 + gr.idx * 128;
-            const unsigned a_lo = p_lo + gr.idx * (kPBytes >> 4), b_lo = v_lo + gr.idx * (kOperand >> 4);
+            const unsigned a_lo = p_lo + gr.idx * (kPBytes >> 4), b_lo = v_lo + vs.idx * (kOperand >> 4);
             const unsigned keep = ((fresh >> gr.idx) & 1u) ^ 1u;
             fresh &= ~(1u << gr.idx);
             if (elect_one()) {
@@ -359,10 +361,12 @@ __device__ void pv_role(const Params &P, Tail *tl, unsigned p_smem, unsigned v_s
                         tc_mma_bf16_split_masked(d_tmem, a_lo + ((s4 * 32) >> 4), kHiK, b_lo + ((tile * kTile + s4 * 2048) >> 4),
                                                  kHiK, kIdescPV, s4 != 0 ? 1u : keep, lo_off, lo_off, hi_off, hi_off);
                 }
-                tc_commit(smem_u32(&tl->o_full[gr.idx]));  // product added = V stage and P buffer of the group free
+                tc_commit(smem_u32(&tl->o_full[gr.idx]));  // product added: the group's P buffer is free
+                tc_commit(smem_u32(&tl->v_empty[vs.idx]));
             }
             __syncwarp();
             gr.advance(2);
+            vs.advance(P.n_v_stages);
         }
         if (elect_one()) mbar_arrive(smem_u32(&tl->m_empty[ms.idx]));
         __syncwarp();
@@ -584,19 +588,21 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
                const __grid_constant__ CUtensorMap tmap_v, Params P) {  // P by value: n_k_stages is filled in here
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char *smem = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    // what is left behind the aligned base decides the number of K stages (the same in every thread)
+    // what is left behind the aligned base decides the number of V and K stages (the same in every thread)
     const int fixed_bytes = (int)(smem - smem_raw) + (int)sizeof(Tail) + kMaskSlots * 2 * P.row_stride * (int)sizeof(int);
-    P.n_k_stages = min(kMaxKStages, (P.smem_bytes - fixed_bytes) / kOperand - kFixedOperands);
+    const int n_rings = (P.smem_bytes - fixed_bytes) / kOperand - kFixedOperands;  // buffers for the two rings: 4 or 5
+    P.n_v_stages = n_rings >= 5 ? 3 : 2;
+    P.n_k_stages = min(kMaxKStages, n_rings - P.n_v_stages);
     const unsigned q_smem = smem_u32(smem), p_smem = q_smem + kOperand, v_smem = p_smem + 2 * kPBytes,
-                   k_smem = v_smem + kVStages * kOperand;
-    Tail *tl = (Tail *)(smem + (kFixedOperands + P.n_k_stages) * kOperand);
+                   k_smem = v_smem + P.n_v_stages * kOperand;
+    Tail *tl = (Tail *)(smem + (kFixedOperands + P.n_v_stages + P.n_k_stages) * kOperand);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
         mbar_init(smem_u32(&tl->q_full), 1);
         mbar_init(smem_u32(&tl->q_empty), 1);
         for (int i = 0; i < kMaxKStages; ++i) { mbar_init(smem_u32(&tl->k_full[i]), 1); mbar_init(smem_u32(&tl->k_empty[i]), 1); }
-        for (int i = 0; i < kVStages; ++i) mbar_init(smem_u32(&tl->v_full[i]), 1);
+        for (int i = 0; i < kMaxVStages; ++i) { mbar_init(smem_u32(&tl->v_full[i]), 1); mbar_init(smem_u32(&tl->v_empty[i]), 1); }
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&tl->s_full[i]), 1); mbar_init(smem_u32(&tl->s_empty[i]), 4);
             mbar_init(smem_u32(&tl->p_full[i]), 4); mbar_init(smem_u32(&tl->o_full[i]), 1);
@@ -668,18 +674,18 @@ stream_status launch_attn_tc(const Geom &g, const void *q, const void *k, const 
     P.scale_log2 = scale * 1.4426950408889634f;
     const int n_sm = sm_count();
     if (n_sm <= 0) { set_error("cannot read the SM count of the current device"); return STREAM_ERR_CUDA; }
-    // room for three K stages if the mask rows are short enough, else two; 1 KB of slack for the
+    // room for five ring buffers (three V, two K) if the mask rows are short enough, else four; 1 KB of slack for the
     // alignment of the base (the kernel counts its stages from what it really gets)
     P.row_stride = (g.k_top + 3) & ~3;
     const int tail_bytes = (int)sizeof(Tail) + kMaskSlots * 2 * P.row_stride * (int)sizeof(int);
-    int smem_bytes = (kFixedOperands + kMaxKStages) * kOperand + tail_bytes + 1024;
+    int smem_bytes = (kFixedOperands + 5) * kOperand + tail_bytes + 1024;
     if (smem_bytes > kMaxSmemPerCta) smem_bytes = kMaxSmemPerCta;
-    if (smem_bytes < (kFixedOperands + 2) * kOperand + tail_bytes + 1024) {
+    if (smem_bytes < (kFixedOperands + 4) * kOperand + tail_bytes + 1024) {
         set_error("tensor-core attention kernel: k_top = %d needs more shared memory than one CTA has", g.k_top);
         return STREAM_ERR_UNSUPPORTED;
     }
     P.smem_bytes = smem_bytes;
-    P.n_k_stages = 0;
+    P.n_k_stages = P.n_v_stages = 0;
     cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmemPerCta);
     if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(attn_tc)");
     const int grid = (int)(n_items < n_sm ? n_items : n_sm);

@@ -221,7 +221,7 @@ def test_attention_tensor_core_non_causal(S):
 
 @pytest.mark.parametrize("impl", ["tensor", "generic"])
 @pytest.mark.parametrize("causal", [True, False])
-@pytest.mark.parametrize("k_top", [6, 200])  # 200: long mask rows leave the tensor-core kernel fewer K stages
+@pytest.mark.parametrize("k_top", [6, 200])  # 200: long mask rows leave the tensor-core kernel four ring buffers instead of five
 def test_attention_arbitrary_mask(S, impl, causal, k_top):
     """Any int32 mask is legal input: unsorted, with holes, rows of unequal length, blocks after the
     query (all their keys are excluded under a causal C), rows with nothing kept (zeros)."""

@@ -44,7 +44,7 @@ typedef enum { STREAM_F32 = 0, STREAM_BF16 = 1 } stream_dtype;
 
 typedef enum {
     STREAM_IMPL_AUTO = 0,    /* tensor-core kernels when the shape allows, else the generic ones */
-    STREAM_IMPL_GENERIC = 1, /* fp32-FMA kernels: any dtype, d in {16,32,64,128}, blocks 1..64 */
+    STREAM_IMPL_GENERIC = 1, /* fp32-FMA kernels: any dtype, d in {16,32,64,128,256}, blocks 1..64 */
     STREAM_IMPL_TENSOR = 2   /* tcgen05 kernels only: bf16, d = 128, block_q = block_k = 64, strides
                                 that are multiples of 8 elements, 16-byte aligned pointers (and
                                 k_top <= 32 for the mask build); otherwise STREAM_ERR_UNSUPPORTED */
@@ -55,7 +55,7 @@ typedef struct {
     int32_t n_q_heads;      /* >= 1 */
     int32_t n_kv_heads;     /* >= 1 and divides n_q_heads */
     int64_t T;              /* tokens, >= 1; need not be a multiple of the block sizes */
-    int32_t d;              /* head dimension */
+    int32_t d;              /* head dimension: 16, 32, 64, 128 or 256 */
     int32_t block_q;        /* b_q */
     int32_t block_k;        /* b_k */
     int32_t k_top;          /* k: key blocks kept per query block = row width of the mask; 1..1024 */

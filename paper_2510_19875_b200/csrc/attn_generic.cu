@@ -149,8 +149,9 @@ stream_status dispatch_d(const Geom &g, const void *q, const void *k, const void
         case 32: return launch<T, 32>(g, qq, kk, vv, mask, scale, (T *)out, st);
         case 64: return launch<T, 64>(g, qq, kk, vv, mask, scale, (T *)out, st);
         case 128: return launch<T, 128>(g, qq, kk, vv, mask, scale, (T *)out, st);
+        case 256: return launch<T, 256>(g, qq, kk, vv, mask, scale, (T *)out, st);
     }
-    set_error("generic attention kernel: head dim %d not in {16, 32, 64, 128}", g.d);
+    set_error("generic attention kernel: head dim %d not in {16, 32, 64, 128, 256}", g.d);
     return STREAM_ERR_UNSUPPORTED;
 }
 

@@ -222,8 +222,9 @@ stream_status dispatch_d(const Geom &g, const MultiK &mk, const void *q, const v
         case 32: return launch<T, 32>(g, mk, qq, kk, mask, score, ws, st);
         case 64: return launch<T, 64>(g, mk, qq, kk, mask, score, ws, st);
         case 128: return launch<T, 128>(g, mk, qq, kk, mask, score, ws, st);
+        case 256: return launch<T, 256>(g, mk, qq, kk, mask, score, ws, st);
     }
-    set_error("generic mask kernel: head dim %d not in {16, 32, 64, 128}", g.d);
+    set_error("generic mask kernel: head dim %d not in {16, 32, 64, 128, 256}", g.d);
     return STREAM_ERR_UNSUPPORTED;
 }
 

@@ -74,6 +74,8 @@ GENERIC_CASES = [
     dict(T=256, k_top=16),                                         # k > N_k: full mask, no levels
     dict(T=64, block=64, k_top=2),                                 # a single key block
     dict(T=1, block=32, k_top=1, n_q_heads=1),                     # one token
+    dict(dtype="bf16", d=256, block=32, T=1500, k_top=4, n_q_heads=4, n_kv_heads=1, sink=True),  # head dim 256
+    dict(d=256, block=64, T=700, k_top=3),                         # head dim 256, fp32
     dict(T=4096, d=64, block=32, k_top=1, n_q_heads=1),            # k = 1: pure binary descent
 ]
 
@@ -184,6 +186,8 @@ def attention_parity(S, w, rows, *, impl="auto", block_q=None, block_k=None, cau
     dict(dtype="bf16", d=128, block=64, T=2048, k_top=8, n_q_heads=4, n_kv_heads=2, sink=True),
     dict(T=777, d=32, block=16, k_top=3, batch=2),
     dict(T=256, k_top=16),
+    dict(dtype="bf16", d=256, block=32, T=1500, k_top=4, n_q_heads=4, n_kv_heads=1, sink=True),
+    dict(d=256, block=64, T=700, k_top=3),
 ])
 def test_attention_generic_small(S, kw):
     w = wl.generate(small_spec(**kw))

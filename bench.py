@@ -31,6 +31,7 @@ if ROOT not in sys.path:
 METRIC = "stream_query_token_heads_per_s"
 UNIT = "query-token-heads/s"
 FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1400.0  # sustained figure of an earlier measurement on this kind of GPU
 
 
 def parse_args():
@@ -127,6 +128,16 @@ def hbm_peak():
             return float(json.load(fh)["hbm_gbs"]), "measured"
     except (OSError, KeyError, ValueError):
         return FALLBACK_HBM_GBS, "fallback"
+
+
+def tensor_peak():
+    """Measured dense bf16 throughput for a kernel timed inside a longer step (TFLOP/s)."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["bf16_tflops_sustained"]), "measured (sustained)"
+    except (OSError, KeyError, ValueError):
+        return FALLBACK_BF16_TFLOPS, "fallback (sustained)"
 
 
 KERNEL_SOURCES = {
@@ -388,6 +399,10 @@ def run_ours(args):
                      "traffic": ncu_traffic(dom["kernel"], spec) if dom["kernel"] in KERNEL_SOURCES and k_row is None else None,
                      "peak_kind": f"of {peak_kind}", "algorithmic_bytes": dom["algorithmic_bytes"],
                      "share_of_step": dom["ms"] / (mask_ms + attn_ms),
+                     # context: the gathers are L2 hits on this part (compare `traffic`), so the same
+                     # launch is also given against the tensor-core peak
+                     "tensor": {"achieved": dom["tensor_tflops"], "peak": tensor_peak()[0], "unit": "TFLOP/s",
+                                "frac": dom["tensor_tflops"] / tensor_peak()[0], "peak_kind": f"of {tensor_peak()[1]}"},
                      "frac_of_8TBs_nominal": dom["algorithmic_gbs"] / 8000.0},
         "clocks": clocks,
         "gpu_launches": 2 * args.steps,

@@ -107,3 +107,29 @@ def test_config3_cot_layer_128k_variable_k_sampled(S):
     report = compare_masks(mask[rows], ora)
     print("variable k", report, "tiles", st.tiles_scored)
     assert report["bad"] == 0, report
+
+
+def test_config3_cot_layer_128k_several_k_sampled(S):
+    """The headline shape with k = 8, 16, 32 in one call (one launch, tile scores shared through
+    the score memory): a row sample of every slab against the oracle."""
+    spec = wl.SPECS["cot_layer_128k"]
+    w = wl.generate(spec)
+    q, k, _ = w.torch_tensors("cuda")
+    ks = [8, 16, 32]
+    res = S.build_masks(q, k, ks, block_q=spec.block, block_k=spec.block)
+    torch.cuda.synchronize()
+    st = res.stats()
+    assert st.error == 0 and st.rows == spec.n_rows * len(ks)
+    assert res.workspace.numel() > 256  # the large workspace: shared scores
+    rows = sample_rows(spec, 1024, seed=11)
+    p = oracle_problem(spec)
+    ora = so.build_mask_rows_multi(p, w.q, w.k, ks, rows, score_cache=True)
+    mask = res.mask.cpu().numpy().reshape(len(ks), -1, spec.k_top)
+    for i, ki in enumerate(ks):
+        check_mask_invariants(mask[i].reshape(1, spec.n_q_heads, spec.n_blocks, spec.k_top)[..., :ki], spec)
+        report = compare_masks(mask[i][rows], {"mask": ora["mask"][i], "min_gap": ora["min_gap"][i]})
+        print("k =", ki, report)
+        assert report["bad"] == 0, (ki, report)
+        assert (mask[i][:, ki:] == -1).all()
+    # sharing: fewer tiles than the largest k alone would need twice over
+    assert st.tiles_scored < 1.05 * 11564329

@@ -497,3 +497,25 @@ def test_mask_tensor_core_repeats_bit_for_bit(S):
             first = (mask, res.scores.cpu().numpy())
         else:
             assert np.array_equal(mask, first[0]) and np.array_equal(res.scores.cpu().numpy(), first[1]), f"launch {it}"
+
+
+def test_several_k_tensor_core_repeats_bit_for_bit(S):
+    """The several-k launch (shared score memory, a group walked once per k) on many short groups
+    of mixed size: ten launches, every slab the oracle's rows every time, and the same tile count."""
+    w = wl.generate(tc_spec(T=2500, k_top=9, n_q_heads=14, n_kv_heads=2, batch=3, local=True))
+    spec = w.spec
+    ks = [3, 9, 5]
+    ora = so.build_mask_rows_multi(oracle_problem(spec), w.q, w.k, ks)
+    q, k, _ = w.torch_tensors("cuda")
+    tiles = None
+    for it in range(10):
+        res = S.build_masks(q, k, ks, block_q=64, block_k=64, impl="tensor")
+        torch.cuda.synchronize()
+        st = res.stats()
+        assert st.error == 0, f"launch {it}: device error {st.error} (info {st.error_info:#x})"
+        mask = res.mask.cpu().numpy().reshape(len(ks), -1, 9)
+        for i in range(len(ks)):
+            ok_rows = ora["min_gap"][i] >= 1e-5
+            assert (mask[i][ok_rows] == ora["mask"][i][ok_rows]).all(), f"launch {it}, k = {ks[i]}"
+        tiles = st.tiles_scored if tiles is None else tiles
+        assert st.tiles_scored == tiles

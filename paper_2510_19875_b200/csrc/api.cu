@@ -156,7 +156,7 @@ static stream_status build_mask_impl(const stream_problem *p, const void *q, con
     WorkspaceHeader *ws = (WorkspaceHeader *)workspace;
     const bool tc_ok = mask_tc_supported(g, p->dtype);
     if (p->impl == STREAM_IMPL_TENSOR && !tc_ok) {
-        set_error("tensor-core mask kernel needs bf16, d = 128, block_q = block_k = 64, k_top <= 64, causal, 16-byte aligned strides");
+        set_error("tensor-core mask kernel needs bf16, d = 128, block_q = block_k = 64, k_top <= 32, more than one key block, 16-byte aligned strides");
         return STREAM_ERR_UNSUPPORTED;
     }
     cudaError_t e = cudaMemsetAsync(ws, 0, sizeof(WorkspaceHeader), st);
@@ -214,7 +214,7 @@ stream_status stream_build_mask_multi(const stream_problem *p, const void *q, co
     WorkspaceHeader *ws = (WorkspaceHeader *)workspace;
     const bool tc_ok = mask_tc_supported(g, p->dtype);
     if (p->impl == STREAM_IMPL_TENSOR && !tc_ok) {
-        set_error("tensor-core mask kernel needs bf16, d = 128, block_q = block_k = 64, k_top <= 32, 16-byte aligned strides");
+        set_error("tensor-core mask kernel needs bf16, d = 128, block_q = block_k = 64, k_top <= 32, more than one key block, 16-byte aligned strides");
         return STREAM_ERR_UNSUPPORTED;
     }
     cudaError_t e = cudaMemsetAsync(ws, 0, sizeof(WorkspaceHeader), st);

@@ -117,15 +117,8 @@ __device__ __forceinline__ void tc_commit(unsigned bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-__device__ __forceinline__ void tc_mma_bf16(unsigned d_tmem, unsigned long long adesc, unsigned long long bdesc,
-                                            unsigned idesc, unsigned accumulate) {
-    asm volatile(
-        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-
-// The same with both descriptors given as (low word, high word). The low word holds the start
+// One tcgen05.mma (kind::f16, cta_group::1): D[tmem] (+)= A[smem] B[smem]. Both shared-memory
+// descriptors are given as (low word, high word): the low word holds the start
 // address in 16-byte units, so a K step is one 32-bit add on it; the high word never changes
 // for a given operand layout.
 __device__ __forceinline__ void tc_mma_bf16_split(unsigned d_tmem, unsigned a_lo, unsigned a_hi, unsigned b_lo,
@@ -172,16 +165,6 @@ __device__ __forceinline__ void tmem_ld_32x32_issue(unsigned taddr, unsigned *r)
         : "r"(taddr)
         : "memory");
 }
-// The same for 16 consecutive columns.
-__device__ __forceinline__ void tmem_ld_32x16_issue(unsigned taddr, unsigned *r) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(taddr)
-        : "memory");
-}
 // Store 32 consecutive fp32 columns of this thread's TMEM lane (the inverse of the load above).
 // Complete for later tcgen05 operations after tmem_st_wait().
 __device__ __forceinline__ void tmem_st_32x32_issue(unsigned taddr, const unsigned *r) {
@@ -216,11 +199,8 @@ __device__ __forceinline__ float warp_max(float x) {
 //   K-major operand (rows of 128 bytes along K): sbo = distance between 8-row groups; lbo unused.
 //   MN-major operand (rows of 128 bytes along M/N, one row per K index): sbo = distance between
 //   8-K-index groups, lbo = distance between consecutive 64-element chunks along M/N.
-__device__ __forceinline__ unsigned long long smem_desc_sw128(unsigned addr, unsigned lbo, unsigned sbo) {
-    return (unsigned long long)((addr >> 4) & 0x3FFF) | ((unsigned long long)((lbo >> 4) & 0x3FFF) << 16) |
-           ((unsigned long long)((sbo >> 4) & 0x3FFF) << 32) | (1ull << 46) | (2ull << 61);
-}
-
+// Bits: start address >> 4 in 0..13, lbo >> 4 in 16..29, sbo >> 4 in 32..45, version 1 in 46..47,
+// swizzle mode 2 (128 bytes) in 61..63.
 // Low and high words of that descriptor; (addr_bytes >> 4) is added to the low word per operand.
 __device__ __forceinline__ unsigned desc_lo_sw128(unsigned addr, unsigned lbo) {
     return ((addr >> 4) & 0x3FFF) | (((lbo >> 4) & 0x3FFF) << 16);

@@ -500,3 +500,17 @@ def test_several_k_at_once_match_the_simulation_and_count_shared_tiles(case):
     assert shared_less  # the k do share representatives
     single = so.build_mask_rows(dataclasses.replace(p, k_top=k_list[-1]), q, kk)["mask"]
     np.testing.assert_array_equal(got["mask"][-1][:, : k_list[-1]], single)
+
+
+@pytest.mark.parametrize("T,blk,s", [(8192, 32, 0.1), (1000, 32, 0.2), (131072, 64, 1 / 128), (4096, 64, 0.5)])
+def test_k_schedule_ends_at_the_papers_formula(T, blk, s):
+    """For the last query block of a causal pattern the row's own count of allowed blocks is
+    ceil(T / b), so the schedule's last entry is the printed k = floor(1 + (T / b_q - 1) s)
+    evaluated with that count (the two agree exactly when b divides T)."""
+    n = -(-T // blk)
+    p = so.OracleProblem(1, 1, 1, T, 2, blk, blk, n, True, "f32")  # k_top = n: no clamp from above
+    got = so.k_schedule(p, s)
+    assert got[-1] == int(math.floor(1 + (n - 1) * s))
+    assert (np.diff(got) >= 0).all() and got[0] == 1  # grows down the pattern, one block at the top
+    if T % blk == 0:
+        assert got[-1] == max(1, min(int(1 + (T / blk - 1) * s), T // blk))

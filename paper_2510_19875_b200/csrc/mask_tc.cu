@@ -5,20 +5,22 @@
 // Candidate key blocks are fetched by TMA (128-byte swizzle) two at a time into a ring of
 // stages; one tcgen05.mma chain per (stage, row) computes K_pair (128 x 128) x Q_row^T (128 x 64)
 // into a 64-column TMEM slot; four epilogue warps reduce the slot to the two masked tile maxima
-// (Eq. 4 under C) - there are two such groups of four, each serving one of every issuing warp's
-// two slots, because the fixed cost of a hand-over (wait, fences, arrive) is larger than the
-// reduction itself and one group alone is the longest stage of the pipeline; a controller warp keeps each row's nodes in registers, ranks the 2k branch
-// scores (higher score, then lower block index), compacts the survivors with ballots and
-// publishes the next level's fetch list. The first level's representatives are the same for
-// every row of a group, so one fetched stage serves all its rows; from the second level on a
-// left branch inherits its parent's score and only right branches are fetched.
+// (Eq. 4 under C). There are two such groups of four, each serving one of every issuing warp's
+// two slots: the fixed cost of a hand-over (wait, fences, arrive) is larger than the reduction
+// itself, and one group alone would be the longest stage of the pipeline. A controller warp keeps
+// each row's nodes in registers, ranks the 2k branch scores (higher score, then lower block
+// index), compacts the survivors with ballots and publishes the next level's fetch list. The
+// first level's representatives are the same for every row of a group, so one fetched stage
+// serves all its rows; from the second level on a left branch inherits its parent's score and
+// only right branches are fetched. With several k per call a group runs the hierarchy once per
+// k on the same Q tiles and fetches only blocks whose score it does not have yet.
 //
 // Roles (512 threads, the last two warps idle): warp 0 TMA producer, warps 1, 3, 12, 13 MMA
 // issuers (warp 1 owns TMEM), warp 2 controller, warps 4..7 and 8..11 the two epilogue groups
-// (TMEM lane quarter = warp % 4). All roles walk the same fixed unit order
-// (level 1: stage-major, row-minor; later levels: row-major), synchronised by mbarriers only.
-// Every wait is bounded: on a timeout the CTA records an error code in the workspace header,
-// raises a shared abort flag, drains its own copies and leaves.
+// (TMEM lane quarter = warp % 4). All roles walk the same fixed unit order (level 1: stage-major,
+// row-minor; later levels: row-major), synchronised by mbarriers only. Every wait is bounded: on
+// a timeout the CTA records an error code in the workspace header, raises a shared abort flag,
+// drains its own copies and leaves.
 #include <math_constants.h>
 
 #include "tc_common.cuh"
@@ -30,7 +32,7 @@ using namespace tc;
 
 constexpr int kThreads = 512;
 constexpr int kEpiGroups = 2;  // group g reduces the chains that land in slot g of their issuing warp
-constexpr int kMmaWarps = 4;   // warps 1, 3, 12, 13 issue the chains in turn
+constexpr int kMmaWarps = 4;   // warps 1, 3, 12, 13 take the stages in turn
 constexpr int kR = 4;          // rows (query heads) per group
 constexpr int kStages = 4;     // K-pair stages
 constexpr int kSlots = 8;      // TMEM accumulator slots of 64 fp32 columns

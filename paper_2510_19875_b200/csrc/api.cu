@@ -367,24 +367,40 @@ stream_status stream_run_host(const stream_problem *p, const void *q_host, const
     STREAM_TRY(cudaStreamWaitEvent(hp->in, hp->start, 0), "cudaStreamWaitEvent");
     STREAM_TRY(cudaStreamWaitEvent(hp->out, hp->start, 0), "cudaStreamWaitEvent");
     const int n_chunks = g.batch * g.G;
+    const size_t q_head = (size_t)g.T * g.d * e, m_head = (size_t)g.n_qb * g.k_top * sizeof(int32_t);
+    int unit = 0;  // running number of the (chunk, heads) units, for the ring of events
     for (int c = 0; c < n_chunks; ++c) {
-        const size_t qo = (size_t)c * q_chunk, ko = (size_t)c * kv_chunk, mo = (size_t)c * m_chunk;
-        cudaEvent_t in_done = hp->in_done[c % kPipeEvents], comp_done = hp->comp_done[c % kPipeEvents];
-        STREAM_TRY(cudaMemcpyAsync(base + s.q + qo, (const char *)q_host + qo, q_chunk, cudaMemcpyHostToDevice, hp->in), "H2D q");
-        STREAM_TRY(cudaMemcpyAsync(base + s.k + ko, (const char *)k_host + ko, kv_chunk, cudaMemcpyHostToDevice, hp->in), "H2D k");
-        STREAM_TRY(cudaMemcpyAsync(base + s.v + ko, (const char *)v_host + ko, kv_chunk, cudaMemcpyHostToDevice, hp->in), "H2D v");
-        STREAM_TRY(cudaEventRecord(in_done, hp->in), "cudaEventRecord");
-        STREAM_TRY(cudaStreamWaitEvent(st, in_done, 0), "cudaStreamWaitEvent");
-        rc = stream_build_mask(&sub, base + s.q + qo, base + s.k + ko, (int32_t *)(base + s.mask + mo), nullptr, base + s.ws,
-                               sizeof(WorkspaceHeader), cuda_stream);
-        if (rc != STREAM_OK) return rc;
-        rc = stream_sparse_attention(&sub, base + s.q + qo, base + s.k + ko, base + s.v + ko,
-                                     (const int32_t *)(base + s.mask + mo), scale, base + s.out + qo, cuda_stream);
-        if (rc != STREAM_OK) return rc;
-        STREAM_TRY(cudaEventRecord(comp_done, st), "cudaEventRecord");
-        STREAM_TRY(cudaStreamWaitEvent(hp->out, comp_done, 0), "cudaStreamWaitEvent");
-        STREAM_TRY(cudaMemcpyAsync((char *)mask_host + mo, base + s.mask + mo, m_chunk, cudaMemcpyDeviceToHost, hp->out), "D2H mask");
-        STREAM_TRY(cudaMemcpyAsync((char *)out_host + qo, base + s.out + qo, q_chunk, cudaMemcpyDeviceToHost, hp->out), "D2H out");
+        const size_t ko = (size_t)c * kv_chunk;
+        // The very last chunk goes through in two halves of its query heads: what is left after the
+        // last byte has arrived (its kernels and its copy out, which nothing overlaps any more) is
+        // then half as long. Everywhere else a chunk keeps all its heads together, so that the
+        // first level's key tiles serve as many rows as possible.
+        const int n_units = (c == n_chunks - 1 && g.hpg >= 4) ? 2 : 1;
+        for (int u = 0; u < n_units; ++u, ++unit) {
+            const int h0 = u * ((g.hpg + n_units - 1) / n_units);
+            const int nh = (u == n_units - 1) ? g.hpg - h0 : (g.hpg + n_units - 1) / n_units;
+            const size_t qo = (size_t)c * q_chunk + (size_t)h0 * q_head, mo = (size_t)c * m_chunk + (size_t)h0 * m_head;
+            const size_t q_bytes = (size_t)nh * q_head, m_bytes = (size_t)nh * m_head;
+            sub.n_q_heads = nh;
+            cudaEvent_t in_done = hp->in_done[unit % kPipeEvents], comp_done = hp->comp_done[unit % kPipeEvents];
+            if (u == 0) {
+                STREAM_TRY(cudaMemcpyAsync(base + s.k + ko, (const char *)k_host + ko, kv_chunk, cudaMemcpyHostToDevice, hp->in), "H2D k");
+                STREAM_TRY(cudaMemcpyAsync(base + s.v + ko, (const char *)v_host + ko, kv_chunk, cudaMemcpyHostToDevice, hp->in), "H2D v");
+            }
+            STREAM_TRY(cudaMemcpyAsync(base + s.q + qo, (const char *)q_host + qo, q_bytes, cudaMemcpyHostToDevice, hp->in), "H2D q");
+            STREAM_TRY(cudaEventRecord(in_done, hp->in), "cudaEventRecord");
+            STREAM_TRY(cudaStreamWaitEvent(st, in_done, 0), "cudaStreamWaitEvent");
+            rc = stream_build_mask(&sub, base + s.q + qo, base + s.k + ko, (int32_t *)(base + s.mask + mo), nullptr, base + s.ws,
+                                   sizeof(WorkspaceHeader), cuda_stream);
+            if (rc != STREAM_OK) return rc;
+            rc = stream_sparse_attention(&sub, base + s.q + qo, base + s.k + ko, base + s.v + ko,
+                                         (const int32_t *)(base + s.mask + mo), scale, base + s.out + qo, cuda_stream);
+            if (rc != STREAM_OK) return rc;
+            STREAM_TRY(cudaEventRecord(comp_done, st), "cudaEventRecord");
+            STREAM_TRY(cudaStreamWaitEvent(hp->out, comp_done, 0), "cudaStreamWaitEvent");
+            STREAM_TRY(cudaMemcpyAsync((char *)mask_host + mo, base + s.mask + mo, m_bytes, cudaMemcpyDeviceToHost, hp->out), "D2H mask");
+            STREAM_TRY(cudaMemcpyAsync((char *)out_host + qo, base + s.out + qo, q_bytes, cudaMemcpyDeviceToHost, hp->out), "D2H out");
+        }
     }
     // the caller's stream is done when the last copy out is
     STREAM_TRY(cudaEventRecord(hp->finish, hp->out), "cudaEventRecord");

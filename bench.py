@@ -48,6 +48,7 @@ def parse_args():
     ap.add_argument("--k-list", default="", help="comma-separated k values: time the several-k mask build (one JSON line, masks only)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true", help="leave the short scaling sweep out of the line")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="target CPU time of the oracle sample")
     ap.add_argument("--sweep", action="store_true",
                     help="instead of the benchmark line: time and peak memory of the sweep workload at every context "
@@ -78,7 +79,7 @@ def workload_config(spec, extra=None):
 
 
 class ClockSampler:
-    """nvidia-smi clocks and throttle reasons, sampled every 200 ms while the timed region runs."""
+    """nvidia-smi clocks and throttle reasons, sampled every 50 ms while the timed region runs."""
 
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
@@ -90,7 +91,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "200"],
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             threading.Thread(target=self._pump, daemon=True).start()
         except OSError:
@@ -158,17 +159,31 @@ def kernel_source_hash(kernel: str) -> str:
 
 
 def ncu_traffic(kernel: str, spec):
-    """DRAM bytes (read + write) per launch of `kernel` on this workload from the committed ncu
-    capture, or None if there is none for this workload and T or the kernel's sources changed since."""
+    """DRAM bytes (read + write) per launch of `kernel` on this workload, from the committed ncu
+    capture of the same workload at a smaller context length, scaled by T: the DRAM traffic of
+    both kernels is their compulsory traffic (Q, K, V in, mask or output out, everything else is
+    served by L2), which grows in proportion to T. None if there is no capture of this workload's
+    shape or the kernel's sources changed since it was taken."""
     path = os.path.join(ROOT, "profiles", "dram_traffic.json")
     try:
         with open(path) as fh:
             rec = json.load(fh)[kernel]
-        if rec["source_hash"] != kernel_source_hash(kernel) or rec["workload"] != spec.name or rec["T"] != spec.T:
+        if rec["source_hash"] != kernel_source_hash(kernel) or rec["workload"] != spec.name:
             return None
-        return float(rec["dram_bytes_per_launch"])
+        return float(rec["dram_bytes_per_launch"]) * spec.T / float(rec["T"])
     except (OSError, KeyError, ValueError):
         return None
+
+
+# Shared-memory traffic per unit of work in the tensor-core kernels' present formulation (bytes that
+# cross the SM's 128-byte-per-clock shared-memory port): what the TMA copies write plus what the
+# tcgen05.mma instructions read as operands.
+#   mask build, per scored tile: the key tile written once (16 KB; shared by the rows of a group at
+#     the first level, counted in full here) + read once as the A operand (16 KB) + the query tile
+#     read as the B operand (8 KB per tile of a two-tile chain)
+#   attention, per kept block: K and V tiles written (32 KB), K and V read as operands (32 KB), the
+#     Q operand (8 KB per block of a two-block chain), P written and read (8 KB + 8 KB)
+SMEM_PORT_BYTES = {"mask_tc_kernel": 40 * 1024, "attn_tc_kernel": 88 * 1024}
 
 
 def rank_env():
@@ -385,6 +400,51 @@ def run_ours(args):
         rec["frac_of_hbm_peak"] = rec["algorithmic_gbs"] / peak
     dominant = max(kernels, key=lambda n: kernels[n]["ms"])
     dom = kernels[dominant]
+    tpeak, tpeak_kind = tensor_peak()
+    n_sm = torch.cuda.get_device_properties(dev).multi_processor_count
+    sm_mhz = (clocks or {}).get("sm_mhz") or 1965.0
+    # Which roof binds the dominant kernel: the time its tile FLOPs need at the measured tensor
+    # peak against the time its compulsory DRAM traffic (every input read once, the result written
+    # once) needs at the measured HBM peak; the larger one is the bound and frac = that time / the
+    # measured time. The gathers of key tiles are served by L2 (compare `traffic`), which is why
+    # the HBM figure on algorithmic bytes is given separately and is not a fraction of a bound.
+    flops = dom["tensor_tflops"] * 1e12 * dom["ms"] * 1e-3
+    compulsory = (units * spec.d * esz + spec.batch * spec.n_kv_heads * spec.T * spec.d * esz + spec.n_rows * spec.k_top * 4
+                  if dominant == "stream_build_mask" else
+                  2 * units * spec.d * esz + 2 * spec.batch * spec.n_kv_heads * spec.T * spec.d * esz + spec.n_rows * spec.k_top * 4)
+    t_tensor_ms = flops / (tpeak * 1e12) * 1e3 if tc else 0.0
+    t_hbm_ms = compulsory / (peak * 1e9) * 1e3
+    traffic = ncu_traffic(dom["kernel"], spec) if dom["kernel"] in KERNEL_SOURCES and k_row is None else None
+    if tc and t_tensor_ms >= t_hbm_ms:
+        roof = {"bound": "tensor", "achieved": dom["tensor_tflops"], "peak": tpeak, "unit": "TFLOP/s",
+                "frac": dom["tensor_tflops"] / tpeak, "peak_kind": f"of {tpeak_kind}"}
+    elif tc or spec.dtype == "bf16":
+        roof = {"bound": "hbm", "achieved": compulsory / (dom["ms"] * 1e-3) / 1e9, "peak": peak, "unit": "GB/s",
+                "frac": t_hbm_ms / dom["ms"], "peak_kind": f"of {peak_kind}"}
+    else:  # the generic kernels: plain fp32 FMA arithmetic
+        alu_peak = n_sm * 128 * 2 * 1.965e9 / 1e12  # SMs x FMA lanes x 2 FLOP x max SM clock
+        roof = {"bound": "alu", "achieved": dom["tensor_tflops"], "peak": alu_peak, "unit": "TFLOP/s",
+                "frac": dom["tensor_tflops"] / alu_peak, "peak_kind": "SMs x 128 FMA lanes x 2 x 1.965 GHz"}
+    roof.update({
+        "kernel": dom["kernel"], "entry_point": dominant, "traffic": traffic,
+        "traffic_kind": "ncu dram bytes of a capture at a smaller T of the same workload, scaled by T (compulsory traffic)",
+        "share_of_step": dom["ms"] / (mask_ms + attn_ms),
+        "bound_times_ms": {"tensor": t_tensor_ms, "hbm_compulsory": t_hbm_ms, "measured": dom["ms"]},
+        # the metric's own accounting: every scored (kept) tile counted as one fetch from memory.
+        # On this GPU those fetches are L2 hits, so this can exceed 1 and is not the binding roof.
+        "hbm_algorithmic": {"achieved": dom["algorithmic_gbs"], "peak": peak, "unit": "GB/s",
+                            "frac": dom["algorithmic_gbs"] / peak, "peak_kind": f"of {peak_kind}",
+                            "algorithmic_bytes": dom["algorithmic_bytes"],
+                            "frac_of_8TBs_nominal": dom["algorithmic_gbs"] / 8000.0,
+                            "note": "served by L2: DRAM carries only `traffic`"},
+    })
+    if dom["kernel"] in SMEM_PORT_BYTES:
+        work = S_tiles if dominant == "stream_build_mask" else kept
+        port_bytes = work * SMEM_PORT_BYTES[dom["kernel"]]
+        port_peak = 128.0 * n_sm * sm_mhz * 1e6 / 1e9  # GB/s at the sampled SM clock
+        roof["smem_port"] = {"model_bytes": port_bytes, "achieved": port_bytes / (dom["ms"] * 1e-3) / 1e9, "peak": port_peak,
+                             "unit": "GB/s", "frac": port_bytes / (dom["ms"] * 1e-3) / 1e9 / port_peak,
+                             "peak_kind": f"128 B/clk x {n_sm} SMs x {sm_mhz:.0f} MHz (sampled)"}
     line = {
         "metric": METRIC, "value": job_value(world, units, args.steps, total_ms), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
@@ -394,24 +454,21 @@ def run_ours(args):
             **({"k_schedule": {"effective_sparsity": args.k_sparsity, "k_min": int(k_row.min()), "k_max": int(k_row.max()),
                                "k_mean": float(k_row.float().mean())}} if k_row is not None else {})}),
         "mask_build": kernels["stream_build_mask"], "sparse_attention": kernels["stream_sparse_attention"],
-        "roofline": {"kernel": dom["kernel"], "entry_point": dominant, "bound": "hbm", "achieved": dom["algorithmic_gbs"],
-                     "peak": peak, "unit": "GB/s", "frac": dom["algorithmic_gbs"] / peak,
-                     "traffic": ncu_traffic(dom["kernel"], spec) if dom["kernel"] in KERNEL_SOURCES and k_row is None else None,
-                     "peak_kind": f"of {peak_kind}", "algorithmic_bytes": dom["algorithmic_bytes"],
-                     "share_of_step": dom["ms"] / (mask_ms + attn_ms),
-                     # context: the gathers are L2 hits on this part (compare `traffic`), so the same
-                     # launch is also given against the tensor-core peak
-                     "tensor": {"achieved": dom["tensor_tflops"], "peak": tensor_peak()[0], "unit": "TFLOP/s",
-                                "frac": dom["tensor_tflops"] / tensor_peak()[0], "peak_kind": f"of {tensor_peak()[1]}"},
-                     "frac_of_8TBs_nominal": dom["algorithmic_gbs"] / 8000.0},
+        "roofline": roof,
         "clocks": clocks,
         "gpu_launches": 2 * args.steps,
     }
     if e2e:
         line["e2e"] = {"value": world * units / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
                        "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"], "steps": e2e["steps"]}
+    del q, k, v, mask
+    if world == 1 and not args.no_sweep:
+        # the scaling sweep's three shortest context lengths (the full sweep is `--sweep`): time and
+        # peak device memory against T, so that "memory linear in T" has a record in this line
+        rows = sweep_rows(wl.SWEEP_T[:3], dev)
+        line["sweep"] = {"rows": [{k2: r[k2] for k2 in ("T", "levels", "mask_ms", "attention_ms", "peak_device_bytes")} for r in rows],
+                         **sweep_fits(rows)}
     if not args.no_cpu_baseline:
-        del q, k, v
         rate, threads, sample = oracle_sample_rate(spec, w, args.cpu_seconds)
         line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample}
     print(json.dumps(line))
@@ -432,10 +489,8 @@ def fit_r2(x, y, through_origin):
     return a, b, 1.0 - ss_res / ss_tot
 
 
-def run_sweep(args):
-    """Scaling of the path with the context length (the paper's complexity ablation, App. A.3): time of
-    both kernels and peak device memory at every T of the sweep workload, and the fits time ~ T (L + 1)
-    (L = levels of the hierarchy, about log2(T / (block k))) and memory ~ T."""
+def sweep_rows(Ts, dev):
+    """Time of both kernels and peak device memory of the sweep workload at each context length in Ts."""
     import math
 
     import torch
@@ -443,14 +498,13 @@ def run_sweep(args):
     from paper_2510_19875_b200 import stream as S
     from paper_2510_19875_b200 import workloads as wl
 
-    dev = torch.device("cuda", 0)
-    torch.cuda.set_device(dev)
     rows = []
-    for T in wl.SWEEP_T:
+    for T in Ts:
         spec = wl.SPECS["sweep"].scaled(T=T)
         w = wl.generate(spec)
         torch.cuda.empty_cache()
         torch.cuda.reset_peak_memory_stats()
+        base = torch.cuda.memory_allocated()
         q, k, v = w.torch_tensors(dev)
         kw = dict(block_q=spec.block, block_k=spec.block, k_top=spec.k_top)
         p = S.make_problem(q, k, **kw)
@@ -473,18 +527,35 @@ def run_sweep(args):
         n_kb = -(-T // spec.block)
         levels = max(1, math.ceil(math.log2(max(1, -(-n_kb // spec.k_top))))) if n_kb > 1 else 0
         rows.append({"T": T, "levels": levels, "mask_ms": best[0], "attention_ms": best[1], "tiles_scored": tiles,
-                     "peak_device_bytes": int(torch.cuda.max_memory_allocated()),
+                     "peak_device_bytes": int(torch.cuda.max_memory_allocated() - base),
                      "input_output_bytes": int((2 * q.numel() + 2 * k.numel()) * q.element_size() + mask.numel() * 4),
                      "workspace_bytes": int(ws.numel())})
         del q, k, v, out, mask, w
+    return rows
+
+
+def sweep_fits(rows):
     Ts = [r["T"] for r in rows]
     a, _, r2_time = fit_r2([r["T"] * (r["levels"] + 1) for r in rows], [r["mask_ms"] for r in rows], True)
     a_lin, _, r2_lin = fit_r2(Ts, [r["mask_ms"] for r in rows], True)
     m_a, m_b, r2_mem = fit_r2(Ts, [r["peak_device_bytes"] for r in rows], False)
-    print(json.dumps({"workload": "sweep", "rows": rows,
-                      "fit_mask_time_vs_T_levels": {"ms_per_token_level": a, "r2": r2_time},
-                      "fit_mask_time_vs_T": {"ms_per_token": a_lin, "r2": r2_lin},
-                      "fit_peak_memory_vs_T": {"bytes_per_token": m_a, "offset_bytes": m_b, "r2": r2_mem}}))
+    return {"fit_mask_time_vs_T_levels": {"ms_per_token_level": a, "r2": r2_time},
+            "fit_mask_time_vs_T": {"ms_per_token": a_lin, "r2": r2_lin},
+            "fit_peak_memory_vs_T": {"bytes_per_token": m_a, "offset_bytes": m_b, "r2": r2_mem}}
+
+
+def run_sweep(args):
+    """Scaling of the path with the context length (the paper's complexity ablation, App. A.3): time of
+    both kernels and peak device memory at every T of the sweep workload, and the fits time ~ T (L + 1)
+    (L = levels of the hierarchy, about log2(T / (block k))) and memory ~ T."""
+    import torch
+
+    from paper_2510_19875_b200 import workloads as wl
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    rows = sweep_rows(wl.SWEEP_T, dev)
+    print(json.dumps({"workload": "sweep", "rows": rows, **sweep_fits(rows)}))
 
 
 def run_k_list(args):

@@ -4,8 +4,11 @@
  *
  * Conventions for every entry point
  *   - Plain C types only. Unless a parameter says HOST, every data pointer is a DEVICE pointer
- *     owned by the caller; the library never allocates or frees device memory and keeps no
- *     state between calls apart from the thread-local error text.
+ *     owned by the caller; the library never allocates or frees device memory. The state it
+ *     keeps between calls is: the thread-local error text; per device, the two copy streams and
+ *     the events of stream_run_host (created at its first call, kept until the process ends);
+ *     per device, the built-in scratch array of stream_build_mask_static and its address; and
+ *     the status word of the tensor-core attention kernel (stream_check_device_status).
  *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = default stream)
  *     and the call returns after enqueue unless stated otherwise.
  *   - Every failure is a returned status; nothing aborts or throws. Arguments are validated on
@@ -103,6 +106,10 @@ size_t stream_workspace_bytes(const stream_problem *p);
  *   score_out  device float32, same shape, or NULL: block score of every kept block, -inf padded
  *   workspace  device, 256-byte aligned, >= stream_workspace_bytes(p); overwritten. After the
  *              stream has drained, stream_read_stats(workspace, ...) returns this call's counters.
+ *              If workspace_bytes >= stream_workspace_bytes(p) + 4 * rows (rows = batch *
+ *              n_q_heads * ceil(T/block_q)), the build also writes, as uint32 [rows] right behind
+ *              the first stream_workspace_bytes(p) bytes, how many tiles each row scored (their
+ *              sum is stream_stats.tiles_scored). stream_build_mask and stream_build_mask_var only.
  *
  * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE before any launch; CUDA if a launch fails.
  */
@@ -162,6 +169,17 @@ stream_status stream_build_mask_multi(const stream_problem *p, const void *q, co
 stream_status stream_k_schedule(const stream_problem *p, double s, int32_t *k_row_host);
 
 /*
+ * The effective-sparsity formula of Section 4.2 as printed: k = floor(1 + (T / b_q - 1) s), kept
+ * inside k's range 1 .. floor(T / b_q) (at least 1). T / b_q is taken as the real quotient. As
+ * printed, a larger s keeps MORE blocks (the prose beside the formula says the opposite; the
+ * formula is followed). Host-only arithmetic; nothing is launched.
+ *
+ *   s           0 <= s <= 1, else INVALID_ARG
+ *   k_out_host  HOST int32, one value
+ */
+stream_status stream_effective_k(int64_t T, int32_t block_q, double s, int32_t *k_out_host);
+
+/*
  * stream_build_mask without a caller-provided workspace and without any allocation. (The paper
  * has no counterpart to this entry point; it exists for deployment.)
  *
@@ -170,7 +188,8 @@ stream_status stream_k_schedule(const stream_problem *p, double s, int32_t *k_ro
  * synchronisation of cudaMalloc / cudaFree. The kernel's scratch (work counter and counters, see
  * stream_stats) lives in a 4096-byte device array built into the library, which each GPU that
  * loads the library holds until the process exits. Same arguments, results and errors as
- * stream_build_mask otherwise; a problem whose scratch need exceeded 4096 bytes would be refused
+ * stream_build_mask otherwise (an invalid or unsupported problem gets exactly the status
+ * stream_build_mask gives it); a problem whose scratch need exceeded 4096 bytes would be refused
  * with STREAM_ERR_WORKSPACE (no current problem does). The call allocates and frees nothing.
  *
  *   - The first call on each device looks up the array's device address (a one-time host-side
@@ -256,6 +275,22 @@ stream_status stream_read_stats(const void *workspace, stream_stats *out, void *
  * bounded waits and left early (its output is then incomplete); STREAM_OK otherwise.
  */
 stream_status stream_check_device_status(void *cuda_stream);
+
+/*
+ * Diagnostic (the paper has no counterpart): runs the bounded wait that every mbarrier wait of the
+ * tensor-core kernels goes through to its limit once, in a one-warp kernel of its own that waits
+ * on a barrier nothing arrives at, with no copy or tensor-core operation in flight. After
+ * limit_cycles SM clock cycles the wait gives up exactly as it would in a product kernel: it
+ * records code 901 in the workspace header, raises the abort flag, all lanes leave together and
+ * the kernel returns. stream_read_stats(workspace, ...) then returns STREAM_ERR_DEVICE_CHECK with
+ * error = 901 (rows = 0: the wait did not succeed; tiles_scored = 1: the abort flag was raised).
+ * The product kernels use the same code path with a limit of 2^31 cycles (about a second).
+ *
+ *   limit_cycles  1 .. 2^31, else INVALID_ARG
+ *   workspace     device, 256-byte aligned, >= 256 bytes; overwritten
+ */
+stream_status stream_selftest_bounded_wait(int64_t limit_cycles, void *workspace, size_t workspace_bytes,
+                                           void *cuda_stream);
 
 /*
  * Bytes of device staging stream_run_host needs: room for Q, K, V, the mask, the output and the

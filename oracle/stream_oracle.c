@@ -385,6 +385,21 @@ int so_k_schedule(const so_problem *p, double s, int32_t *k_row_out) {
 }
 
 /*
+ * The effective-sparsity formula of Section 4.2 as it is printed, applied once to the whole
+ * context: k = floor(1 + (T / b_q - 1) s) with T / b_q the real quotient, kept inside k's range
+ * 1 .. floor(T / b_q) (Section 3), and never below 1. Returns k, or a negative code.
+ */
+int64_t so_effective_k(int64_t T, int64_t block_q, double s) {
+    if (T < 1 || block_q < 1 || !(s >= 0.0 && s <= 1.0)) return -2;
+    const double n = (double)T / (double)block_q;
+    int64_t k = (int64_t)floor(1.0 + (n - 1.0) * s);
+    const int64_t k_max = T / block_q;
+    if (k > k_max) k = k_max;
+    if (k < 1) k = 1;
+    return k;
+}
+
+/*
  * Eq. 2 on block masks: for every query token of each listed row, softmax over the keys of the
  * row's selected blocks that C allows, then the weighted sum of V, all in fp64.
  *   mask [n_rows, k]  as produced above; out [n_rows, b_q, d] fp64; tokens beyond T or with no

@@ -107,6 +107,8 @@ def _load():
         lib.so_build_mask_rows_multi.restype = ctypes.c_int
         lib.so_build_mask_rows_multi.argtypes = [ctypes.POINTER(_CProblem), vp, vp, ctypes.c_int32, vp, i64p,
                                                  ctypes.c_int64, vp, vp, vp, vp, ctypes.c_int]
+        lib.so_effective_k.restype = ctypes.c_int64
+        lib.so_effective_k.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_double]
         lib.so_k_schedule.restype = ctypes.c_int
         lib.so_k_schedule.argtypes = [ctypes.POINTER(_CProblem), ctypes.c_double, vp]
         lib.so_sparse_attention_rows.restype = ctypes.c_int
@@ -232,6 +234,14 @@ def k_schedule(p: OracleProblem, s: float) -> np.ndarray:
     if rc:
         raise RuntimeError(f"so_k_schedule failed with {rc}")
     return out
+
+
+def effective_k(T: int, block_q: int, s: float) -> int:
+    """The printed effective-sparsity formula (Section 4.2): ``floor(1 + (T / b_q - 1) s)`` in 1 .. floor(T / b_q)."""
+    k = int(_load().so_effective_k(int(T), int(block_q), float(s)))
+    if k < 0:
+        raise ValueError("need T, block_q >= 1 and 0 <= s <= 1")
+    return k
 
 
 def sparse_attention_rows(p: OracleProblem, q: np.ndarray, k: np.ndarray, v: np.ndarray, mask: np.ndarray,

@@ -1,42 +1,71 @@
-"""Builds libstream.so (sm_100a) in-tree with nvcc. Run as ``python -m paper_2510_19875_b200.build``."""
+"""Builds libstream.so (sm_100a) in-tree with nvcc. Run as ``python -m paper_2510_19875_b200.build``.
+
+Every source is compiled to an object of its own (in parallel; an object is rebuilt only when its
+source, a header or this file is newer), then the objects are linked into the shared library.
+"""
 from __future__ import annotations
 
 import os
 import subprocess
 import sys
+from concurrent.futures import ThreadPoolExecutor
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
+OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libstream.so")
-SOURCES = ["api.cu", "mask_generic.cu", "attn_generic.cu", "mask_tc.cu", "attn_tc.cu", "static_scratch.cu", "vertical.cu", "mask_diff.cu"]
+SOURCES = ["api.cu", "mask_generic.cu", "attn_generic.cu", "mask_tc.cu", "attn_tc.cu",
+           "static_scratch.cu", "vertical.cu", "mask_diff.cu", "selftest.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "-Xcompiler", "-fPIC", "-shared", "-Xptxas", "-v",
+    "-Xcompiler", "-fPIC", "-Xptxas", "-v",
 ]
 
 
-def _stale() -> bool:
-    if not os.path.exists(LIB):
+def _headers():
+    return [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cuh", ".h"))] + [
+        os.path.join(ROOT, "include", "stream.h"), __file__]
+
+
+def _newer(deps, target) -> bool:
+    if not os.path.exists(target):
         return True
-    t = os.path.getmtime(LIB)
-    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(ROOT, "include", "stream.h"), __file__]
+    t = os.path.getmtime(target)
     return any(os.path.getmtime(d) > t for d in deps)
 
 
 def build_library(force: bool = False, verbose: bool = False) -> str:
-    """Compile every CUDA source into ``libstream.so`` next to this file; returns its path."""
-    if not force and not _stale():
-        return LIB
+    """Compile every CUDA source and link ``libstream.so`` next to this file; returns its path."""
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    cmd = [nvcc, *NVCC_FLAGS, "-I", os.path.join(ROOT, "include"), "-I", CSRC,
-           *[os.path.join(CSRC, s) for s in SOURCES], "-o", LIB + ".tmp"]
-    res = subprocess.run(cmd, capture_output=True, text=True)
-    if verbose or res.returncode != 0:
-        sys.stderr.write(res.stdout + res.stderr)
-    if res.returncode != 0:
-        raise RuntimeError("nvcc failed building libstream.so")
-    os.replace(LIB + ".tmp", LIB)
+    os.makedirs(OBJ, exist_ok=True)
+    headers = _headers()
+    jobs = []
+    for src in SOURCES:
+        path, obj = os.path.join(CSRC, src), os.path.join(OBJ, src[:-3] + ".o")
+        if force or _newer([path, *headers], obj):
+            jobs.append((src, [nvcc, *NVCC_FLAGS, "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-c", path, "-o", obj]))
+
+    def run(job):
+        return job[0], subprocess.run(job[1], capture_output=True, text=True)
+
+    failed = []
+    with ThreadPoolExecutor(max_workers=min(8, max(1, len(jobs)))) as pool:
+        for src, res in pool.map(run, jobs):
+            if verbose or res.returncode != 0:
+                sys.stderr.write(f"--- {src}\n{res.stdout}{res.stderr}")
+            if res.returncode != 0:
+                failed.append(src)
+    if failed:
+        raise RuntimeError("nvcc failed on " + ", ".join(failed))
+    objs = [os.path.join(OBJ, s[:-3] + ".o") for s in SOURCES]
+    if force or jobs or _newer(objs, LIB):
+        res = subprocess.run([nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", *objs, "-o", LIB + ".tmp"],
+                             capture_output=True, text=True)
+        if res.returncode != 0:
+            sys.stderr.write(res.stdout + res.stderr)
+            raise RuntimeError("linking libstream.so failed")
+        os.replace(LIB + ".tmp", LIB)
     return LIB
 
 

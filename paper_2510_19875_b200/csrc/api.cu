@@ -65,6 +65,7 @@ stream_status make_geom(const stream_problem *p, Geom *g) {
     g->levels = levels_for((int)N_k, p->k_top);
     g->k_row = nullptr;
     g->k_override = 0;
+    g->row_tiles = nullptr;
     g->qs_b = p->q_stride_b; g->qs_h = p->q_stride_h; g->qs_t = p->q_stride_t;
     g->ks_b = p->kv_stride_b; g->ks_h = p->kv_stride_h; g->ks_t = p->kv_stride_t;
     return STREAM_OK;
@@ -161,6 +162,9 @@ static stream_status build_mask_impl(const stream_problem *p, const void *q, con
     }
     cudaError_t e = cudaMemsetAsync(ws, 0, sizeof(WorkspaceHeader), st);
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(workspace)");
+    // room behind the header for one counter per row: the build also says how many tiles each row scored
+    const size_t n_rows = (size_t)g.batch * g.H * g.n_qb;
+    if (workspace_bytes >= sizeof(WorkspaceHeader) + n_rows * sizeof(unsigned int)) g.row_tiles = (unsigned int *)(ws + 1);
     if (tc_ok && p->impl != STREAM_IMPL_GENERIC) return launch_mask_tc(g, q, k, mask_out, score_out, ws, st);
     return launch_mask_generic(g, p->dtype, q, k, mask_out, score_out, ws, st);
 }
@@ -253,6 +257,19 @@ stream_status stream_k_schedule(const stream_problem *p, double s, int32_t *k_ro
         long long kq = (long long)floor(1.0 + (double)(n - 1) * s);
         k_row_host[qb] = (int32_t)(kq < 1 ? 1 : (kq > g.k_top ? g.k_top : kq));
     }
+    return STREAM_OK;
+}
+
+stream_status stream_effective_k(int64_t T, int32_t block_q, double s, int32_t *k_out_host) {
+    if (k_out_host == nullptr) { set_error("k_out_host must not be NULL"); return STREAM_ERR_INVALID_ARG; }
+    if (T < 1 || block_q < 1) { set_error("T and block_q must be positive"); return STREAM_ERR_INVALID_ARG; }
+    if (!(s >= 0.0 && s <= 1.0)) { set_error("effective sparsity must lie in [0, 1] (got %g)", s); return STREAM_ERR_INVALID_ARG; }
+    const double n = (double)T / (double)block_q;            // T / b_q as the formula has it (not rounded)
+    const long long n_rows = T / block_q > 1 ? T / block_q : 1;  // floor(T / b_q), the upper end of k's range
+    long long kq = (long long)floor(1.0 + (n - 1.0) * s);
+    kq = kq < 1 ? 1 : (kq > n_rows ? n_rows : kq);
+    if (kq > 0x7fffffffLL) { set_error("k does not fit 32 bits"); return STREAM_ERR_UNSUPPORTED; }
+    *k_out_host = (int32_t)kq;
     return STREAM_OK;
 }
 

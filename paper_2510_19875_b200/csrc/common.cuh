@@ -18,6 +18,7 @@ struct Geom {
     int levels;                 // split levels that can change the result (with k = k_top)
     const int32_t *k_row;       // device, [n_qb]: k of each query block (clamped to 1 .. k_top), or NULL = k_top everywhere
     int k_override;             // > 0: every row uses this k (one launch of a several-k build); rows stay k_top wide
+    unsigned int *row_tiles;    // device, [batch * H * n_qb] or NULL: tiles scored for each row (single-k builds)
     long long qs_b, qs_h, qs_t; // element strides
     long long ks_b, ks_h, ks_t;
 };

@@ -192,6 +192,7 @@ __global__ void __launch_bounds__(kThreads) mask_generic_kernel(Geom g, MultiK m
     if (tid == 0) {
         atomicAdd(&ws->tiles_scored, (unsigned long long)tiles);
         atomicAdd(&ws->rows, 1ull);
+        if (g.row_tiles != nullptr) g.row_tiles[row] = tiles;
     }
 }
 

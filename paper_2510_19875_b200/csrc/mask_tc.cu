@@ -401,9 +401,13 @@ __device__ void controller_role(const Params &P, Tail *tl, int lane) {
             float ns[kR], cs[kR];
             bool has_r[kR], need[kR];
             unsigned tiles = 0;  // (row, block) tiles that had no score yet
+            unsigned rt[kR];     // the same, row by row
 #pragma unroll
-            for (int r = 0; r < kR; ++r)
-                if (r < R) tiles += (unsigned)(__popc(__ballot_sync(0xffffffffu, (miss_l >> r) & 1u)) + __popc(__ballot_sync(0xffffffffu, (miss_r >> r) & 1u)));
+            for (int r = 0; r < kR; ++r) {
+                rt[r] = 0;
+                if (r < R) rt[r] = (unsigned)(__popc(__ballot_sync(0xffffffffu, (miss_l >> r) & 1u)) + __popc(__ballot_sync(0xffffffffu, (miss_r >> r) & 1u)));
+                tiles += rt[r];
+            }
             for (int level = 0; level < levels; ++level) {
 #pragma unroll
                 for (int r = 0; r < kR; ++r) {
@@ -458,6 +462,7 @@ __device__ void controller_role(const Params &P, Tail *tl, int lane) {
                         if (need[r]) tl->jobs_blk[r][my_c[r]] = rb[r];
                         if (lane == 0) tl->n_jobs[r] = __popc(hb);
                         tiles += (unsigned)__popc(hb);
+                        rt[r] += (unsigned)__popc(hb);
                         __syncwarp();
                         if (lane == 0) mbar_arrive(smem_u32(&tl->jobs_ready[r]));
                     } else {
@@ -467,6 +472,8 @@ __device__ void controller_role(const Params &P, Tail *tl, int lane) {
                             P.mask[o + lane] = live ? nf[r] : -1;
                             if (P.score != nullptr) P.score[o + lane] = live ? ns[r] : -CUDART_INF_F;
                         }
+                        if (!kMulti && g.row_tiles != nullptr && lane == 0)
+                            g.row_tiles[((long long)b * g.H + (h0 + r)) * g.n_qb + qb] = rt[r];
                     }
                 }
             }

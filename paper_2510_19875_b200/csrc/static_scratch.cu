@@ -47,7 +47,9 @@ extern "C" stream_status stream_build_mask_static(const stream_problem *p, const
                                                   int32_t *mask_out, float *score_out, void *cuda_stream) {
     using namespace stream;
     const size_t need = stream_workspace_bytes(p);
-    if (need == 0) return STREAM_ERR_INVALID_ARG;  // text set by the validation
+    // 0: the problem is invalid or unsupported. The workspace variant validates the problem before it
+    // looks at its workspace, so asking it gives exactly the status (and text) it would give.
+    if (need == 0) return stream_build_mask(p, q, k, mask_out, score_out, nullptr, 0, cuda_stream);
     if (need > kStaticScratchBytes) {
         set_error("this problem needs %zu bytes of scratch, the built-in array holds %zu: use stream_build_mask with a workspace",
                   need, kStaticScratchBytes);
@@ -57,5 +59,6 @@ extern "C" stream_status stream_build_mask_static(const stream_problem *p, const
     stream_status rc = scratch_for_current_device(&scratch);
     if (rc != STREAM_OK) return rc;
     // Same path as the workspace variant from here on; it zeroes the header on the stream first.
-    return stream_build_mask(p, q, k, mask_out, score_out, scratch, kStaticScratchBytes, cuda_stream);
+    // (Just the header's bytes are handed over, which keeps the optional per-row counters off.)
+    return stream_build_mask(p, q, k, mask_out, score_out, scratch, need, cuda_stream);
 }

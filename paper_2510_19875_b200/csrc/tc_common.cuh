@@ -58,12 +58,12 @@ __device__ __forceinline__ bool mbar_test_wait(unsigned bar, unsigned parity) {
 // out, in which case it raises the CTA's abort flag and records `code` (first one wins) with the
 // block index in the two error words.
 static __device__ __noinline__ bool mbar_wait_slow(unsigned bar, unsigned parity, int *abort_flag, unsigned *err_code,
-                                                   unsigned *err_info, unsigned code) {
+                                                   unsigned *err_info, unsigned code, long long limit) {
     const long long t0 = clock64();
     for (;;) {
         if (mbar_try_wait_suspend(bar, parity, 4000u)) return true;
         if (*(volatile int *)abort_flag) return false;
-        if (clock64() - t0 > kWaitCycles) {
+        if (clock64() - t0 > limit) {
             *(volatile int *)abort_flag = 1;
             if (atomicCAS(err_code, 0u, code) == 0u) *err_info = blockIdx.x;
             return false;
@@ -71,9 +71,9 @@ static __device__ __noinline__ bool mbar_wait_slow(unsigned bar, unsigned parity
     }
 }
 __device__ __forceinline__ bool mbar_wait_bounded(unsigned bar, unsigned parity, int *abort_flag, unsigned *err_code,
-                                                  unsigned *err_info, unsigned code) {
+                                                  unsigned *err_info, unsigned code, long long limit = kWaitCycles) {
     if (mbar_try_wait(bar, parity)) return true;  // the common case costs one instruction
-    return mbar_wait_slow(bar, parity, abort_flag, err_code, err_info, code);
+    return mbar_wait_slow(bar, parity, abort_flag, err_code, err_info, code, limit);
 }
 
 // True in exactly one lane of a converged warp (the same lane every time).
@@ -87,8 +87,8 @@ __device__ __forceinline__ bool elect_one() {
 // answer (false as soon as one lane saw the abort flag or ran out of time), so that the warp
 // stays converged for the elect_one() that follows.
 __device__ __forceinline__ bool mbar_wait_warp(unsigned bar, unsigned parity, int *abort_flag, unsigned *err_code,
-                                               unsigned *err_info, unsigned code) {
-    const bool ok = mbar_wait_bounded(bar, parity, abort_flag, err_code, err_info, code);
+                                               unsigned *err_info, unsigned code, long long limit = kWaitCycles) {
+    const bool ok = mbar_wait_bounded(bar, parity, abort_flag, err_code, err_info, code, limit);
     return __all_sync(0xffffffffu, ok);
 }
 

@@ -82,6 +82,10 @@ def _load():
     lib.stream_build_mask_multi.argtypes = [P, vp, vp, ctypes.c_int32, vp, vp, vp, vp, sz, vp]
     lib.stream_k_schedule.restype = ctypes.c_int
     lib.stream_k_schedule.argtypes = [P, ctypes.c_double, vp]
+    lib.stream_effective_k.restype = ctypes.c_int
+    lib.stream_effective_k.argtypes = [ctypes.c_int64, ctypes.c_int32, ctypes.c_double, ctypes.POINTER(ctypes.c_int32)]
+    lib.stream_selftest_bounded_wait.restype = ctypes.c_int
+    lib.stream_selftest_bounded_wait.argtypes = [ctypes.c_int64, vp, sz, vp]
     lib.stream_build_mask_static.restype = ctypes.c_int
     lib.stream_build_mask_static.argtypes = [P, vp, vp, vp, vp, vp]
     lib.stream_sparse_attention.restype = ctypes.c_int
@@ -166,6 +170,18 @@ def stream_k_schedule(p: StreamProblem, s: float, k_row_host) -> None:
     _raise(_load().stream_k_schedule(ctypes.byref(p), float(s), _addr(k_row_host)))
 
 
+def stream_effective_k(T: int, block_q: int, s: float) -> int:
+    """k for an effective sparsity ``s`` (the printed formula of Section 4.2, computed by the library)."""
+    out = ctypes.c_int32(0)
+    _raise(_load().stream_effective_k(int(T), int(block_q), float(s), ctypes.byref(out)))
+    return int(out.value)
+
+
+def stream_selftest_bounded_wait(limit_cycles: int, workspace, workspace_bytes: int, stream=None) -> None:
+    """Diagnostic kernel whose bounded wait runs out after ``limit_cycles``; read the outcome with stream_read_stats."""
+    _raise(_load().stream_selftest_bounded_wait(int(limit_cycles), _addr(workspace), workspace_bytes, _stream_handle(stream)))
+
+
 def stream_build_mask_static(p: StreamProblem, q, k, mask_out, score_out, stream=None) -> None:
     """Mask build on the library's built-in scratch: no workspace argument, nothing allocated."""
     _raise(_load().stream_build_mask_static(ctypes.byref(p), _addr(q), _addr(k), _addr(mask_out), _addr(score_out),
@@ -236,37 +252,50 @@ class MaskResult:
     mask: torch.Tensor            # int32 [B, H, n_query_blocks, k_top]
     scores: torch.Tensor | None   # float32, same shape, if requested
     workspace: torch.Tensor       # holds the counters of this call; see stream_read_stats
+    header_bytes: int = 256       # stream_workspace_bytes of the problem: optional per-row counters sit behind it
 
     def stats(self, stream=None) -> StreamStats:
         return stream_read_stats(self.workspace, stream)
 
+    def row_tiles(self) -> torch.Tensor | None:
+        """int32 [B, H, n_query_blocks]: tiles scored per row, if the workspace had room for them."""
+        rows = self.mask.shape[0] * self.mask.shape[1] * self.mask.shape[2]
+        if self.mask.dim() != 4 or self.workspace.numel() < self.header_bytes + 4 * rows:
+            return None
+        return self.workspace[self.header_bytes:self.header_bytes + 4 * rows].view(torch.int32).view(self.mask.shape[:3])
 
-def new_workspace(p: StreamProblem, device) -> torch.Tensor:
+
+def new_workspace(p: StreamProblem, device, row_tiles: bool = False) -> torch.Tensor:
+    """Workspace of the size the library asks for; with ``row_tiles`` also room for one counter per row."""
     n = stream_workspace_bytes(p)
     if n == 0:
         raise StreamError(STREAM_ERR_INVALID_ARG, stream_last_error())
+    if row_tiles:
+        n += 4 * p.batch * p.n_q_heads * n_query_blocks(p)
     return torch.empty(n, dtype=torch.uint8, device=device)
 
 
 def build_mask(q: torch.Tensor, k: torch.Tensor, *, block_q: int, block_k: int, k_top: int, causal: bool = True,
                impl: str = "auto", want_scores: bool = False, mask_out: torch.Tensor | None = None,
-               workspace: torch.Tensor | None = None, k_row: torch.Tensor | None = None, stream=None) -> MaskResult:
+               workspace: torch.Tensor | None = None, k_row: torch.Tensor | None = None, row_tiles: bool = False,
+               stream=None) -> MaskResult:
     """Mask of every row. With ``k_row`` (int32 CUDA tensor, one k per query block, see
-    :func:`k_schedule`) each row uses its own k and ``k_top`` is the row width."""
+    :func:`k_schedule`) each row uses its own k and ``k_top`` is the row width. ``row_tiles``
+    makes the workspace large enough for the per-row tile counters (``MaskResult.row_tiles()``)."""
     if not q.is_cuda or not k.is_cuda:
         raise ValueError("q and k must be CUDA tensors (there is no CPU path)")
     p = make_problem(q, k, block_q=block_q, block_k=block_k, k_top=k_top, causal=causal, impl=impl)
     shape = (p.batch, p.n_q_heads, n_query_blocks(p), k_top)
     mask = mask_out if mask_out is not None else torch.empty(shape, dtype=torch.int32, device=q.device)
     scores = torch.empty(shape, dtype=torch.float32, device=q.device) if want_scores else None
-    ws = workspace if workspace is not None else new_workspace(p, q.device)
+    ws = workspace if workspace is not None else new_workspace(p, q.device, row_tiles)
     if k_row is None:
         stream_build_mask(p, q, k, mask, scores, ws, ws.numel(), stream)
     else:
         if not k_row.is_cuda or k_row.dtype != torch.int32 or not k_row.is_contiguous() or tuple(k_row.shape) != (shape[2],):
             raise ValueError(f"k_row must be a contiguous int32 CUDA tensor of shape ({shape[2]},)")
         stream_build_mask_var(p, q, k, k_row, mask, scores, ws, ws.numel(), stream)
-    return MaskResult(mask, scores, ws)
+    return MaskResult(mask, scores, ws, stream_workspace_bytes(p))
 
 
 def build_masks(q: torch.Tensor, k: torch.Tensor, k_list, *, block_q: int, block_k: int, causal: bool = True,
@@ -357,10 +386,6 @@ def mask_difference(mask_a: torch.Tensor, mask_b: torch.Tensor, scores_a: torch.
 
 
 def effective_k(T: int, block_q: int, s: float) -> int:
-    """Sparsity constant for an effective sparsity ``s`` in [0, 1] (Section 4.2 of the paper):
-    ``k = floor(1 + (T / b_q - 1) s)``, kept inside ``1 .. floor(T / b_q)``. As printed, a larger
-    ``s`` keeps MORE blocks (the prose beside the formula says the opposite; the formula is followed)."""
-    if T < 1 or block_q < 1:
-        raise ValueError("T and block_q must be positive")
-    n = T / block_q
-    return max(1, min(int(1 + (n - 1) * s), max(1, T // block_q)))
+    """Sparsity constant for an effective sparsity ``s`` in [0, 1] (Section 4.2 of the paper), as
+    computed by the library's ``stream_effective_k``."""
+    return stream_effective_k(T, block_q, s)

@@ -108,10 +108,32 @@ def test_staging_size_covers_all_buffers(S):
 
 
 def test_effective_k_follows_the_printed_formula(S):
+    """stream_effective_k (host-only arithmetic inside the library) against hand values and the oracle."""
+    from oracle import stream_oracle as so
+
     assert S.effective_k(1000, 32, 0.0) == 1
     assert S.effective_k(1000, 32, 1.0) == 31          # floor(T / b_q)
     assert S.effective_k(8192, 32, 0.1) == 26           # floor(1 + 255 * 0.1)
     assert S.effective_k(64, 64, 0.5) == 1
+    for T in (1, 63, 64, 1000, 4096, 131072, 1048576):
+        for bq in (1, 32, 64):
+            for s in (0.0, 0.01, 0.04, 0.25, 0.5, 0.99, 1.0):
+                assert S.stream_effective_k(T, bq, s) == so.effective_k(T, bq, s), (T, bq, s)
+    for args in ((0, 32, 0.5), (100, 0, 0.5), (100, 32, -0.1), (100, 32, 1.01), (100, 32, float("nan"))):
+        with pytest.raises(S.StreamError) as e:
+            S.stream_effective_k(*args)
+        assert e.value.status == S.STREAM_ERR_INVALID_ARG
+
+
+def test_selftest_wait_rejects_bad_arguments_on_the_host(S):
+    for limit in (0, -5, (1 << 31) + 1):
+        with pytest.raises(S.StreamError) as e:
+            S.stream_selftest_bounded_wait(limit, 256, 256, stream=0)
+        assert e.value.status == S.STREAM_ERR_INVALID_ARG
+    for ws, n in ((None, 256), (256, 128), (264, 256)):
+        with pytest.raises(S.StreamError) as e:
+            S.stream_selftest_bounded_wait(1000, ws, n, stream=0)
+        assert e.value.status == S.STREAM_ERR_WORKSPACE
 
 
 @pytest.mark.parametrize("kw,s", [

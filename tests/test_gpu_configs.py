@@ -14,10 +14,10 @@ from test_gpu_parity import ATTN_TOL, S  # noqa: F401  (fixture)
 pytestmark = pytest.mark.gpu
 
 
-def run_config(S, spec, n_rows, n_attn_rows=64):
+def run_config(S, spec, n_rows, n_attn_rows=None):
     w = wl.generate(spec)
     q, k, v = w.torch_tensors("cuda")
-    res = S.build_mask(q, k, block_q=spec.block, block_k=spec.block, k_top=spec.k_top)
+    res = S.build_mask(q, k, block_q=spec.block, block_k=spec.block, k_top=spec.k_top, row_tiles=True)
     torch.cuda.synchronize()
     st = res.stats()
     assert st.error == 0 and st.rows == spec.n_rows
@@ -29,8 +29,14 @@ def run_config(S, spec, n_rows, n_attn_rows=64):
     report = compare_masks(mask.reshape(-1, spec.k_top)[rows], ora)
     print(spec.name, spec.T, report, "tiles", st.tiles_scored)
     assert report["bad"] == 0, report
-    # attention on a subsample, with the oracle's mask on both sides
-    sub = rows[:: max(1, len(rows) // n_attn_rows)]
+    # the counter the roofline figures rest on: the total is the sum over the rows, and every
+    # sampled row that is not a near-tie scored exactly the oracle's distinct tiles
+    rt = res.row_tiles().cpu().numpy().reshape(-1).astype(np.int64)
+    assert int(rt.sum()) == st.tiles_scored
+    agree = (mask.reshape(-1, spec.k_top)[rows] == ora["mask"]).all(axis=1) & (ora["min_gap"] >= 1e-5)
+    assert (rt[rows][agree] == ora["tiles"][agree]).all()
+    # attention on the sampled rows (all of them unless told otherwise), with the oracle's mask on both sides
+    sub = rows if n_attn_rows is None else rows[:: max(1, len(rows) // n_attn_rows)]
     full = np.full((spec.n_rows, spec.k_top), -1, np.int32)
     full[rows] = ora["mask"]
     mask_dev = torch.from_numpy(full.reshape(mask.shape)).cuda()
@@ -80,7 +86,7 @@ def test_config4_needle_stack_32k_sampled(S):
 def test_config5_sweep(S, T):
     spec = wl.SPECS["sweep"].scaled(T=T)
     n = spec.n_rows if T <= 16384 else (1024 if T <= 262144 else 384)
-    run_config(S, spec, n, n_attn_rows=32)
+    run_config(S, spec, n, n_attn_rows=1024)
 
 
 def test_config3_cot_layer_128k_variable_k_sampled(S):

@@ -26,7 +26,7 @@ def run_mask(S, w, *, impl="auto", block_q=None, block_k=None, k_top=None, causa
     spec = w.spec
     q, k, _ = w.torch_tensors("cuda")
     res = S.build_mask(q, k, block_q=block_q or spec.block, block_k=block_k or spec.block,
-                       k_top=k_top or spec.k_top, causal=causal, impl=impl, want_scores=want_scores)
+                       k_top=k_top or spec.k_top, causal=causal, impl=impl, want_scores=want_scores, row_tiles=True)
     torch.cuda.synchronize()
     return res
 
@@ -52,10 +52,13 @@ def assert_mask_parity(S, w, rows, *, impl="auto", score_cache=True, **kw):
     np.testing.assert_allclose(sc[same][fin], ora["scores"][same][fin], rtol=2e-5, atol=2e-5)
     assert (sc[same][~fin] == -np.inf).all()
     assert st.rows == flat.shape[0]
-    if rows is None:
-        agree = same & (ora["min_gap"] >= 1e-5)
-        if agree.all():
-            assert st.tiles_scored == int(ora["tiles"].sum())
+    # tiles scored, row by row: every row that is not a near-tie must have scored exactly the
+    # oracle's distinct (row, representative block) tiles; the total is the sum of the rows
+    rt = res.row_tiles().cpu().numpy().reshape(-1).astype(np.int64)
+    assert int(rt.sum()) == st.tiles_scored
+    rt = rt if rows is None else rt[rows]
+    agree = same & (ora["min_gap"] >= 1e-5)
+    assert (rt[agree] == ora["tiles"][agree]).all()
     return report
 
 
@@ -115,7 +118,9 @@ def test_mask_tensor_core_non_causal(S):
     assert_mask_parity(S, w, None, impl="tensor", score_cache=False, causal=False)
 
 
-def test_mask_tensor_core_matches_generic_kernel(S):
+def test_consistency_of_the_two_mask_kernels(S):
+    """Not a parity test (each kernel is compared with the oracle above): the two CUDA kernels
+    against each other, as a cheap cross-check that they count and score the same tiles."""
     w = wl.generate(tc_spec(T=8192, k_top=16, n_q_heads=8, n_kv_heads=2, anchors=True))
     a = run_mask(S, w, impl="tensor", want_scores=True)
     b = run_mask(S, w, impl="generic", want_scores=True)
@@ -517,3 +522,20 @@ def test_several_k_tensor_core_repeats_bit_for_bit(S):
             assert (mask[i][ok_rows] == ora["mask"][i][ok_rows]).all(), f"launch {it}, k = {ks[i]}"
         tiles = st.tiles_scored if tiles is None else tiles
         assert st.tiles_scored == tiles
+
+
+def test_a_bounded_wait_that_runs_out_is_reported(S):
+    """The diagnostic kernel waits on a barrier nothing arrives at; after its limit the wait gives
+    up the way every wait of the tensor-core kernels would: error word, abort flag, the warp
+    leaves together, the kernel returns, and the host reads STREAM_ERR_DEVICE_CHECK. The context
+    stays usable: a mask build right after it gives the oracle's rows."""
+    ws = torch.empty(256, dtype=torch.uint8, device="cuda")
+    S.stream_selftest_bounded_wait(1_000_000, ws, ws.numel())   # about half a millisecond
+    with pytest.raises(S.StreamError) as e:
+        S.stream_read_stats(ws)
+    assert e.value.status == S.STREAM_ERR_DEVICE_CHECK
+    words = ws.cpu().numpy().view(np.uint64)
+    assert words[0] == 1 and words[1] == 0          # abort flag raised; the wait did not succeed
+    assert ws.cpu().numpy().view(np.uint32)[4] == 901
+    w = wl.generate(tc_spec(T=2048, k_top=4))
+    assert_mask_parity(S, w, None, impl="tensor", score_cache=False)

@@ -28,10 +28,15 @@ def test_static_scratch_entry_point_matches_workspace_entry_point_twice():
         for _ in range(2):
             mask = torch.full_like(ref.mask, -7)
             scores = torch.zeros_like(ref.scores)
+            torch.cuda.synchronize()
             before = torch.cuda.memory_allocated()
+            # the driver's own count of free bytes sees what torch's allocator cannot: a cudaMalloc
+            # inside the library. (The kernels' code was loaded by the workspace calls above.)
+            free_before = torch.cuda.mem_get_info()[0]
             S.stream_build_mask_static(p, q, k, mask, scores)
             torch.cuda.synchronize()
             assert torch.cuda.memory_allocated() == before
+            assert torch.cuda.mem_get_info()[0] >= free_before
             assert torch.equal(mask, ref.mask)       # masks are integer work: bit-exact
             assert torch.equal(scores, ref.scores)   # same kernel, same inputs: same fp32 scores
 
@@ -45,3 +50,12 @@ def test_static_scratch_entry_point_validates_like_the_other():
     with pytest.raises(S.StreamError) as e:
         S.stream_build_mask_static(p, q, q, q, None)
     assert e.value.status == S.STREAM_ERR_INVALID_ARG
+    # a valid request that no kernel covers: the same status from both entry points
+    p = S.make_problem(q, q, block_q=32, block_k=32, k_top=2)
+    p.k_top = 2000
+    ws = torch.empty(256, dtype=torch.uint8, device="cuda")
+    for call in (lambda: S.stream_build_mask_static(p, q, q, q, None),
+                 lambda: S.stream_build_mask(p, q, q, q, None, ws, ws.numel())):
+        with pytest.raises(S.StreamError) as e:
+            call()
+        assert e.value.status == S.STREAM_ERR_UNSUPPORTED

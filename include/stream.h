@@ -50,7 +50,9 @@ typedef enum {
     STREAM_IMPL_GENERIC = 1, /* fp32-FMA kernels: any dtype, d in {16,32,64,128,256}, blocks 1..64 */
     STREAM_IMPL_TENSOR = 2   /* tcgen05 kernels only: bf16, d = 128, block_q = block_k = 64, strides
                                 that are multiples of 8 elements, 16-byte aligned pointers (and
-                                k_top <= 32 for the mask build); otherwise STREAM_ERR_UNSUPPORTED */
+                                k_top <= 32 for the mask build); the mask build also takes
+                                block_q = 1 (per-token masks) with block_k = 64, one k, and at most
+                                32768 key blocks; otherwise STREAM_ERR_UNSUPPORTED */
 } stream_impl;
 
 typedef struct {
@@ -75,6 +77,10 @@ typedef struct {
     uint64_t rows;         /* rows finished */
     uint32_t error;        /* 0, or a code saying which bounded wait ran out (kernel returned early) */
     uint32_t error_info;
+    uint64_t tile_products; /* 64 x 64 x d tile products the per-token tensor-core kernel computed (it
+                               multiplies every fetched key tile with 128 tokens at once, so this
+                               exceeds tiles_scored / 64); 0 from the other kernels, whose products
+                               are exactly the tiles scored */
 } stream_stats;
 
 /* Library version: major * 10000 + minor * 100 + patch. */

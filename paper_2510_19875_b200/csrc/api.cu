@@ -155,9 +155,10 @@ static stream_status build_mask_impl(const stream_problem *p, const void *q, con
     }
     cudaStream_t st = (cudaStream_t)cuda_stream;
     WorkspaceHeader *ws = (WorkspaceHeader *)workspace;
-    const bool tc_ok = mask_tc_supported(g, p->dtype);
-    if (p->impl == STREAM_IMPL_TENSOR && !tc_ok) {
-        set_error("tensor-core mask kernel needs bf16, d = 128, block_q = block_k = 64, k_top <= 32, more than one key block, 16-byte aligned strides");
+    const bool tc_ok = mask_tc_supported(g, p->dtype), tok_ok = mask_tok_supported(g, p->dtype);
+    if (p->impl == STREAM_IMPL_TENSOR && !tc_ok && !tok_ok) {
+        set_error("tensor-core mask kernels need bf16, d = 128, block_k = 64, block_q = 64 or (with one k and at most 32768 key "
+                  "blocks) 1, k_top <= 32, more than one key block, 16-byte aligned strides");
         return STREAM_ERR_UNSUPPORTED;
     }
     cudaError_t e = cudaMemsetAsync(ws, 0, sizeof(WorkspaceHeader), st);
@@ -166,6 +167,7 @@ static stream_status build_mask_impl(const stream_problem *p, const void *q, con
     const size_t n_rows = (size_t)g.batch * g.H * g.n_qb;
     if (workspace_bytes >= sizeof(WorkspaceHeader) + n_rows * sizeof(unsigned int)) g.row_tiles = (unsigned int *)(ws + 1);
     if (tc_ok && p->impl != STREAM_IMPL_GENERIC) return launch_mask_tc(g, q, k, mask_out, score_out, ws, st);
+    if (tok_ok && p->impl != STREAM_IMPL_GENERIC) return launch_mask_tok(g, q, k, mask_out, score_out, ws, st);
     return launch_mask_generic(g, p->dtype, q, k, mask_out, score_out, ws, st);
 }
 

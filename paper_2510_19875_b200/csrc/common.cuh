@@ -23,14 +23,15 @@ struct Geom {
     long long ks_b, ks_h, ks_t;
 };
 
-// Header at the start of the mask workspace. The first 24 bytes mirror stream_stats.
+// Header at the start of the mask workspace. The first 32 bytes mirror stream_stats.
 struct WorkspaceHeader {
     unsigned long long tiles_scored;
     unsigned long long rows;
     unsigned int error;
     unsigned int error_info;
+    unsigned long long tile_products;  // 64 x 64 tile products computed (more than tiles_scored where rows share a product)
     unsigned int work_counter;  // next work item of the persistent kernels
-    unsigned int pad[57];
+    unsigned int pad[55];
 };
 static_assert(sizeof(WorkspaceHeader) == 256, "workspace header is 256 bytes");
 
@@ -63,6 +64,10 @@ stream_status launch_mask_tc(const Geom &g, const void *q, const void *k, int32_
 size_t mask_tc_score_memory_bytes(const Geom &g);
 stream_status launch_mask_tc_multi(const Geom &g, const MultiK &mk, const void *q, const void *k, int32_t *mask,
                                    float *score, WorkspaceHeader *ws, void *score_memory, cudaStream_t st);
+// Per-token masks (block_q = 1) on the tensor cores.
+bool mask_tok_supported(const Geom &g, int dtype);
+stream_status launch_mask_tok(const Geom &g, const void *q, const void *k, int32_t *mask, float *score,
+                              WorkspaceHeader *ws, cudaStream_t st);
 bool attn_tc_supported(const Geom &g, int dtype);
 stream_status launch_attn_tc(const Geom &g, const void *q, const void *k, const void *v, const int32_t *mask,
                              float scale, void *out, cudaStream_t st);

@@ -302,26 +302,7 @@ __device__ void epilogue_role(const Params &P, Tail *tl, unsigned tmem_base, int
     }
 }
 
-// Controller helpers -----------------------------------------------------------------------------
-struct Keep { bool l, r; };
-
-// Rank the (up to) 64 candidates held two per lane; keep the k best by (score desc, index asc).
-__device__ __forceinline__ Keep select_topk(bool vl, float sl, bool vr, float sr, int k, int lane) {
-    const int total = __popc(__ballot_sync(0xffffffffu, vl)) + __popc(__ballot_sync(0xffffffffu, vr));
-    if (total <= k) return {vl, vr};
-    const float el = vl ? sl : -CUDART_INF_F, er = vr ? sr : -CUDART_INF_F;
-    int rank_l = 0, rank_r = 0;
-#pragma unroll 8
-    for (int j = 0; j < 32; ++j) {
-        const float ol = __shfl_sync(0xffffffffu, el, j), orr = __shfl_sync(0xffffffffu, er, j);
-        rank_l += (ol > el) || (ol == el && j < lane);
-        rank_l += (orr > el) || (orr == el && j < lane);
-        rank_r += (ol > er) || (ol == er && j <= lane);
-        rank_r += (orr > er) || (orr == er && j < lane);
-    }
-    return {vl && rank_l < k, vr && rank_r < k};
-}
-
+// Controller ----------------------------------------------------------------------------------------
 // kMulti: several k per group with the score memory; false compiles the plain single-pass
 // controller (its ranking step is on every group's critical path, so it carries nothing extra).
 template <bool kMulti>

@@ -212,6 +212,27 @@ __host__ __device__ constexpr unsigned idesc_bf16(unsigned M, unsigned N, bool b
     return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((N >> 3) << 17) | ((M >> 4) << 24);
 }
 
+// Top-k of the (up to) 64 candidates a warp holds two per lane (a node's left and right branch):
+// keep the k best by (score descending, candidate index ascending), the candidates numbered
+// 2 * lane (left) and 2 * lane + 1 (right). Rank by counting, with shuffles.
+struct Keep { bool l, r; };
+__device__ __forceinline__ Keep select_topk(bool vl, float sl, bool vr, float sr, int k, int lane) {
+    const int total = __popc(__ballot_sync(0xffffffffu, vl)) + __popc(__ballot_sync(0xffffffffu, vr));
+    if (total <= k) return {vl, vr};
+    const float ninf = __int_as_float(0xff800000);
+    const float el = vl ? sl : ninf, er = vr ? sr : ninf;
+    int rank_l = 0, rank_r = 0;
+#pragma unroll 8
+    for (int j = 0; j < 32; ++j) {
+        const float ol = __shfl_sync(0xffffffffu, el, j), orr = __shfl_sync(0xffffffffu, er, j);
+        rank_l += (ol > el) || (ol == el && j < lane);
+        rank_l += (orr > el) || (orr == el && j < lane);
+        rank_r += (ol > er) || (ol == er && j <= lane);
+        rank_r += (orr > er) || (orr == er && j < lane);
+    }
+    return {vl && rank_l < k, vr && rank_r < k};
+}
+
 struct Ring {  // position in a ring of barriers with phase tracking
     int idx = 0;
     unsigned phase = 0;
@@ -239,10 +260,10 @@ inline EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// [batch, heads, T, 128] bf16 with element strides -> 4-D map with a 64 x 64 box, 128-byte swizzle.
-// Rows beyond T read as zeros.
+// [batch, heads, T, 128] bf16 with element strides -> 4-D map with a box of 64 channels x box_rows
+// tokens (64 unless told otherwise), 128-byte swizzle. Rows beyond T read as zeros.
 inline stream_status make_map_bf16_d128(CUtensorMap *map, const void *base, long long T, int heads, int batch,
-                                        long long s_t, long long s_h, long long s_b, const char *what) {
+                                        long long s_t, long long s_h, long long s_b, const char *what, int box_rows = 64) {
     EncodeTiledFn fn = encode_fn();
     if (fn == nullptr) { set_error("cuTensorMapEncodeTiled is not available from this driver"); return STREAM_ERR_CUDA; }
     // extents of 1 may come with arbitrary strides: give them a well-formed one
@@ -250,7 +271,7 @@ inline stream_status make_map_bf16_d128(CUtensorMap *map, const void *base, long
     if (batch == 1) s_b = s_h * heads;
     cuuint64_t dims[4] = {128, (cuuint64_t)T, (cuuint64_t)heads, (cuuint64_t)batch};
     cuuint64_t strides[3] = {(cuuint64_t)s_t * 2, (cuuint64_t)s_h * 2, (cuuint64_t)s_b * 2};
-    cuuint32_t box[4] = {64, 64, 1, 1}, estr[4] = {1, 1, 1, 1};
+    cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1}, estr[4] = {1, 1, 1, 1};
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);

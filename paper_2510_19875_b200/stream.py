@@ -40,7 +40,7 @@ class StreamStats(ctypes.Structure):
     """``stream_stats`` of stream.h."""
 
     _fields_ = [("tiles_scored", ctypes.c_uint64), ("rows", ctypes.c_uint64), ("error", ctypes.c_uint32),
-                ("error_info", ctypes.c_uint32)]
+                ("error_info", ctypes.c_uint32), ("tile_products", ctypes.c_uint64)]
 
 
 class StreamError(RuntimeError):

@@ -139,3 +139,35 @@ def test_config3_cot_layer_128k_several_k_sampled(S):
         assert (mask[i][:, ki:] == -1).all()
     # sharing: fewer tiles than the largest k alone would need twice over
     assert st.tiles_scored < 1.05 * 11564329
+
+
+@pytest.mark.parametrize("name,T", [("gqa_layer_16k", 16384), ("cot_layer_128k", 131072)])
+def test_per_token_masks_at_layer_size(S, name, T):
+    """block_q = 1 (a mask row for every query token, the [heads, T, k] shape) on the layer shapes
+    with 32 / 8 heads, through the tensor-core per-token kernel: a seeded sample of token rows
+    against the oracle (the first and last tokens of the first and last head always included),
+    the size-independent invariants and the per-row tile counts on every sampled row."""
+    spec = wl.SPECS[name].scaled(T=T)
+    w = wl.generate(spec, with_v=False)
+    q, k, _ = w.torch_tensors("cuda")
+    res = S.build_mask(q, k, block_q=1, block_k=spec.block, k_top=spec.k_top, row_tiles=True)
+    torch.cuda.synchronize()
+    st = res.stats()
+    n_rows = spec.n_q_heads * T
+    assert st.error == 0 and st.rows == n_rows
+    assert st.tile_products > 0   # the per-token tensor-core kernel ran, not the generic one
+    mask = res.mask.cpu().numpy()
+    check_mask_invariants(mask, spec, block_q=1, block_k=spec.block)
+    rng = np.random.default_rng(spec.seed)
+    edge = [h * T + t for h in (0, spec.n_q_heads - 1) for t in list(range(130)) + list(range(T - 130, T))]
+    rows = np.unique(np.concatenate([np.array(edge, np.int64), rng.choice(n_rows, size=4096, replace=False)]))
+    p = oracle_problem(spec, block_q=1, block_k=spec.block)
+    ora = so.build_mask_rows(p, w.q, w.k, rows, score_cache=True)
+    got = mask.reshape(-1, spec.k_top)[rows]
+    report = compare_masks(got, ora)
+    print("per-token", name, T, report, "tiles", st.tiles_scored, "products", st.tile_products)
+    assert report["bad"] == 0, report
+    rt = res.row_tiles().cpu().numpy().reshape(-1).astype(np.int64)
+    assert int(rt.sum()) == st.tiles_scored
+    agree = (got == ora["mask"]).all(axis=1) & (ora["min_gap"] >= 1e-5)
+    assert (rt[rows][agree] == ora["tiles"][agree]).all()

@@ -137,6 +137,42 @@ def test_mask_generic_unequal_blocks(S, bq, bk):
     assert_mask_parity(S, w, None, impl="generic", score_cache=False, block_q=bq, block_k=bk)
 
 
+TOKEN_CASES = [
+    dict(T=2048, k_top=4),                                        # 32 key blocks, three levels, 16 groups of 128 tokens
+    dict(T=1000, k_top=5, n_q_heads=3, n_kv_heads=1),             # ragged T (last group and last key block partial), odd k
+    dict(T=4096, k_top=8, n_q_heads=4, n_kv_heads=2, anchors=True),
+    dict(T=3000, k_top=32, n_q_heads=2, n_kv_heads=2),            # k close to N_k: one level
+    dict(T=8192, k_top=1, n_q_heads=1, n_kv_heads=1),             # k = 1: binary descent per token
+    dict(T=700, k_top=3, batch=2, n_q_heads=2, n_kv_heads=1, local=True),
+    dict(T=130, k_top=2),                                         # three key blocks, two groups
+]
+
+
+@pytest.mark.parametrize("kw", TOKEN_CASES)
+def test_mask_per_token_tensor_core_small(S, kw):
+    """block_q = 1 (every token a row of its own) on the tensor-core path, every row against the oracle."""
+    w = wl.generate(tc_spec(**kw))
+    assert_mask_parity(S, w, None, impl="tensor", score_cache=False, block_q=1, block_k=64)
+
+
+def test_mask_per_token_tensor_core_non_causal(S):
+    w = wl.generate(tc_spec(T=1500, k_top=6, n_q_heads=2, n_kv_heads=1))
+    assert_mask_parity(S, w, None, impl="tensor", score_cache=False, block_q=1, block_k=64, causal=False)
+
+
+def test_mask_per_token_tensor_core_repeats_and_matches_generic(S):
+    w = wl.generate(tc_spec(T=3000, k_top=7, n_q_heads=4, n_kv_heads=2, anchors=True))
+    a = run_mask(S, w, impl="tensor", block_q=1, block_k=64, want_scores=True)
+    for _ in range(3):
+        b = run_mask(S, w, impl="tensor", block_q=1, block_k=64, want_scores=True)
+        assert torch.equal(a.mask, b.mask) and torch.equal(a.scores, b.scores)
+        assert a.stats().tiles_scored == b.stats().tiles_scored
+    c = run_mask(S, w, impl="generic", block_q=1, block_k=64)   # consistency only: both are checked against the oracle
+    assert (a.mask == c.mask).all(-1).float().mean().item() > 0.97
+    st = a.stats()
+    assert st.tile_products >= st.tiles_scored // 64              # every needed tile is inside a computed product
+
+
 def test_mask_generic_non_causal(S):
     w = wl.generate(small_spec(T=900, k_top=6, n_q_heads=2, n_kv_heads=2))
     assert_mask_parity(S, w, None, impl="generic", score_cache=False, causal=False)

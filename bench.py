@@ -46,6 +46,8 @@ def parse_args():
     ap.add_argument("--k-sparsity", type=float, default=0.0,
                     help="build the mask with k per query block from this effective sparsity (0 = one k; implies --no-e2e)")
     ap.add_argument("--k-list", default="", help="comma-separated k values: time the several-k mask build (one JSON line, masks only)")
+    ap.add_argument("--block-q", type=int, default=0,
+                    help="1: time the per-token mask build (block_q = 1, masks only) instead of the step")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="leave the short scaling sweep out of the line")
@@ -588,8 +590,90 @@ def run_k_list(args):
     print(json.dumps(out))
 
 
+def run_per_token(args):
+    """The per-token mask build (block_q = 1, block_k = the workload's block): one step = one
+    stream_build_mask call on the workload's Q and K (masks only: the attention pass for
+    per-token masks runs on the generic kernel and is not part of this line)."""
+    import torch
+
+    from paper_2510_19875_b200 import stream as S
+    from paper_2510_19875_b200 import workloads as wl
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    spec = get_spec(args, 0)
+    w = wl.generate(spec, with_v=False)
+    q, k, _ = w.torch_tensors(dev)
+    p = S.make_problem(q, k, block_q=1, block_k=spec.block, k_top=spec.k_top, impl=args.kernels)
+    mask = torch.empty((spec.batch, spec.n_q_heads, spec.T, spec.k_top), dtype=torch.int32, device=dev)
+    ws = S.new_workspace(p, dev)
+    stream = torch.cuda.current_stream()
+    for _ in range(args.warmup):
+        S.stream_build_mask(p, q, k, mask, None, ws, ws.numel(), stream)
+    sampler = ClockSampler(0)
+    sampler.start()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    a.record()
+    for _ in range(args.steps):
+        S.stream_build_mask(p, q, k, mask, None, ws, ws.numel(), stream)
+    b.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = a.elapsed_time(b) / args.steps
+    st = S.stream_read_stats(ws, stream)
+    units = spec.batch * spec.n_q_heads * spec.T
+    esz = 2 if spec.dtype == "bf16" else 4
+    tile_flops = 2.0 * 64 * 64 * spec.d
+    tpeak, tpeak_kind = tensor_peak()
+    peak, peak_kind = hbm_peak()
+    products = int(st.tile_products)
+    on_tensor = products > 0
+    achieved = products * tile_flops / (ms * 1e-3) / 1e12
+    compulsory = units * spec.d * esz + spec.batch * spec.n_kv_heads * spec.T * spec.d * esz + units * spec.k_top * 4
+    line = {
+        "metric": METRIC, "value": units / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": spec.dtype,
+        "data": "synthetic",
+        "config": workload_config(spec, {"block_q": 1, "kernels": args.kernels, "step": "per-token mask build only",
+                                         "l2": "inputs larger than L2" if (q.numel() + k.numel()) * esz > 126e6 else "inputs fit L2"}),
+        "mask_build": {"kernel": "mask_tok_kernel" if on_tensor else "mask_generic_kernel", "ms": ms,
+                       "tiles_scored": int(st.tiles_scored), "tile_products": products,
+                       "useful_fraction_of_products": (int(st.tiles_scored) / 64.0) / products if products else None},
+        "roofline": {"bound": "tensor", "kernel": "mask_tok_kernel", "entry_point": "stream_build_mask", "achieved": achieved,
+                     "peak": tpeak, "unit": "TFLOP/s", "frac": achieved / tpeak, "peak_kind": f"of {tpeak_kind}", "traffic": None,
+                     "flops": "tile products the kernel computed (every fetched key tile x 128 tokens) x 2 x 64 x 64 x d",
+                     "bound_times_ms": {"tensor": products * tile_flops / (tpeak * 1e12) * 1e3,
+                                        "hbm_compulsory": compulsory / (peak * 1e9) * 1e3, "measured": ms}} if on_tensor else None,
+        "clocks": clocks, "gpu_launches": args.steps, "e2e": None,
+    }
+    if not args.no_cpu_baseline:
+        import numpy as np
+
+        from oracle import stream_oracle as so
+
+        op = so.OracleProblem(spec.batch, spec.n_q_heads, spec.n_kv_heads, spec.T, spec.d, 1, spec.block, spec.k_top, True, spec.dtype)
+        rng = np.random.default_rng(1234)
+        n = 64 * so.threads()
+        t_cpu = 0.0
+        while True:
+            rows = np.sort(rng.choice(units, size=min(n, units), replace=False))
+            t0 = time.perf_counter()
+            so.build_mask_rows(op, w.q, w.k, rows)
+            t_cpu = time.perf_counter() - t0
+            if t_cpu > args.cpu_seconds / 3 or n >= units:
+                break
+            n = int(n * max(2.0, args.cpu_seconds / max(t_cpu, 1e-3) * 0.7))
+        line["cpu_baseline"] = {"value": len(rows) / t_cpu, "unit": UNIT, "cores": so.threads(), "kind": "oracle",
+                                "sample": f"{len(rows)} seeded token rows of {units} (mask only), {t_cpu:.1f} s wall"}
+    print(json.dumps(line))
+
+
 def main():
     args = parse_args()
+    if args.block_q == 1:
+        run_per_token(args)
+        return
     if args.k_list:
         run_k_list(args)
         return

@@ -56,7 +56,7 @@ constexpr int kPBytes = 2 * kHalfTile;      // one group's P: 128 rows x 64 keys
 constexpr int kMaxKStages = 3, kMaxVStages = 3;
 constexpr int kMaskSlots = 2;               // pairs whose mask rows are resident
 constexpr int kMaxKTopTc = 1024;
-constexpr float kLazyLog2 = 8.f;            // ref is raised when the maximum exceeds it by this much (log2 units)
+constexpr float kLazySum = 68719476736.f;   // 2^36 = 64 * 2^30: the 64 P of an entry add up to more only if one of them exceeds 2^30 (its logit has outgrown the reference by 30 in log2 units)
 
 // TMEM columns: S of group g at 128 g, O of group g at 256 + 128 g.
 struct Tail {
@@ -284,7 +284,7 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
                 }
             }
             if (__shfl_sync(0xffffffffu, stop, 0)) return;
-            __nanosleep(64);  // leave the issue slots to the softmax warps of this scheduler
+            __nanosleep(200);  // leave the issue slots to the softmax warps of this scheduler
         }
     }
 }
@@ -381,12 +381,6 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 
-__device__ __forceinline__ float max3(float a, float b, float c) {
-    float y;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
-    return y;
-}
-
 // Multiplies 128 fp32 columns of this thread's TMEM lane by f, in place (every lane of the warp
 // takes part; lanes that need no change pass f = 1).
 __device__ __forceinline__ void rescale_lane(unsigned taddr, float f) {
@@ -456,24 +450,50 @@ __device__ void softmax_role(const Params &P, Tail *tl, unsigned char *p_ptr, un
                 n_hi = (int)max(0ll, min(lim, (long long)kBlk));
             }
             const bool all_keys = n_hi == kBlk;  // every block but the diagonal one and the one across T
-            float mx4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
-            if (all_keys) {
+            // P = exp2(scale (s - ref)) under the token's current reference, their sum, the packed row.
+            // No reference yet (+inf shift: any allowed logit then gives +inf) or a logit that has
+            // outgrown the reference by more than kLazyLog2 both show in the sum of the 64 P, which
+            // is needed anyway: the maximum itself is only taken when that happens.
+            unsigned packed[32];
+            float esum;
+            auto make_p = [&](float shift) {
+                float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+                if (all_keys) {
 #pragma unroll
-                for (int i = 0; i < 64; i += 8) {
-                    mx4[0] = max3(mx4[0], __uint_as_float(sr[i]), __uint_as_float(sr[i + 1]));
-                    mx4[1] = max3(mx4[1], __uint_as_float(sr[i + 2]), __uint_as_float(sr[i + 3]));
-                    mx4[2] = max3(mx4[2], __uint_as_float(sr[i + 4]), __uint_as_float(sr[i + 5]));
-                    mx4[3] = max3(mx4[3], __uint_as_float(sr[i + 6]), __uint_as_float(sr[i + 7]));
+                    for (int i = 0; i < 64; i += 2) {
+                        const float p0 = fast_exp2(fmaf(__uint_as_float(sr[i]), P.scale_log2, shift));
+                        const float p1 = fast_exp2(fmaf(__uint_as_float(sr[i + 1]), P.scale_log2, shift));
+                        sum4[(i >> 1) & 3] += p0 + p1;
+                        __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+                        packed[i >> 1] = *reinterpret_cast<unsigned *>(&pk);
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 64; i += 2) {
+                        float p0 = fast_exp2(fmaf(__uint_as_float(sr[i]), P.scale_log2, shift));
+                        float p1 = fast_exp2(fmaf(__uint_as_float(sr[i + 1]), P.scale_log2, shift));
+                        p0 = i < n_hi ? p0 : 0.f;
+                        p1 = i + 1 < n_hi ? p1 : 0.f;
+                        sum4[(i >> 1) & 3] += p0 + p1;
+                        __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+                        packed[i >> 1] = *reinterpret_cast<unsigned *>(&pk);
+                    }
                 }
-            } else {
+                esum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+            };
+            auto masked_max = [&]() {
+                float mx = -CUDART_INF_F;
 #pragma unroll
-                for (int i = 0; i < 64; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], i < n_hi ? __uint_as_float(sr[i]) : -CUDART_INF_F);
+                for (int i = 0; i < 64; ++i) mx = fmaxf(mx, i < n_hi ? __uint_as_float(sr[i]) : -CUDART_INF_F);
+                return mx;
+            };
+            // the token's first allowed logits set its reference (once per pair)
+            if (__any_sync(0xffffffffu, ref == -CUDART_INF_F && n_hi > 0)) {
+                const float mx = masked_max();
+                if (ref == -CUDART_INF_F) ref = mx;
             }
-            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-            // the reference: the first allowed logits set it; later it only moves when the maximum
-            // has outgrown it by kLazyLog2, and then what the group has accumulated is rescaled
-            const bool raise = ref != -CUDART_INF_F && (mx - ref) * P.scale_log2 > kLazyLog2;
-            const float new_ref = (ref == -CUDART_INF_F || raise) ? mx : ref;
+            make_p(ref == -CUDART_INF_F ? 0.f : -ref * P.scale_log2);
+            const bool redo = !(esum <= kLazySum);
             // this group's previous chain of the pair must be done before its P buffer is rewritten
             // or its O lane rescaled
             if (pending) {
@@ -481,37 +501,19 @@ __device__ void softmax_role(const Params &P, Tail *tl, unsigned char *p_ptr, un
                 o_par ^= 1;
                 tc_fence_after();
             }
-            if (__any_sync(0xffffffffu, raise)) {
-                const float f = raise ? fast_exp2((ref - new_ref) * P.scale_log2) : 1.f;
+            if (__any_sync(0xffffffffu, redo)) {  // rare: a logit has outgrown the token's reference
+                const float mx = masked_max();
+                float f = 1.f;
+                if (redo) {
+                    f = fast_exp2((ref - mx) * P.scale_log2);
+                    ref = mx;
+                }
+                // what the group has accumulated for this token is brought to the new reference
                 rescale_lane(o_own, f);
                 l *= f;
+                if (redo) make_p(-ref * P.scale_log2);
             }
-            ref = new_ref;
-            const float shift = ref == -CUDART_INF_F ? 0.f : -ref * P.scale_log2;
-            float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-            unsigned packed[32];
-            if (all_keys) {
-#pragma unroll
-                for (int i = 0; i < 64; i += 2) {
-                    const float p0 = fast_exp2(fmaf(__uint_as_float(sr[i]), P.scale_log2, shift));
-                    const float p1 = fast_exp2(fmaf(__uint_as_float(sr[i + 1]), P.scale_log2, shift));
-                    sum4[(i >> 1) & 3] += p0 + p1;
-                    __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
-                    packed[i >> 1] = *reinterpret_cast<unsigned *>(&pk);
-                }
-            } else {
-#pragma unroll
-                for (int i = 0; i < 64; i += 2) {
-                    float p0 = fast_exp2(fmaf(__uint_as_float(sr[i]), P.scale_log2, shift));
-                    float p1 = fast_exp2(fmaf(__uint_as_float(sr[i + 1]), P.scale_log2, shift));
-                    p0 = i < n_hi ? p0 : 0.f;
-                    p1 = i + 1 < n_hi ? p1 : 0.f;
-                    sum4[(i >> 1) & 3] += p0 + p1;
-                    __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
-                    packed[i >> 1] = *reinterpret_cast<unsigned *>(&pk);
-                }
-            }
-            l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+            l += esum;
 #pragma unroll
             for (int c = 0; c < 8; ++c)
                 *reinterpret_cast<uint4 *>(p_row + ((c ^ sw) << 4)) =

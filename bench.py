@@ -48,6 +48,9 @@ def parse_args():
     ap.add_argument("--k-list", default="", help="comma-separated k values: time the several-k mask build (one JSON line, masks only)")
     ap.add_argument("--block-q", type=int, default=0,
                     help="1: time the per-token mask build (block_q = 1, masks only) instead of the step")
+    ap.add_argument("--extras", action="store_true",
+                    help="instead of the benchmark line: time the analysis kernels (vertical scores, mask subtraction) and "
+                         "the several-k build on the workload's masks, each against the HBM peak (one JSON object)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="leave the short scaling sweep out of the line")
@@ -669,8 +672,76 @@ def run_per_token(args):
     print(json.dumps(line))
 
 
+def run_extras(args):
+    """The kernels around the mask: vertical scores + kurtosis (binary and score-weighted), mask
+    subtraction (k against k / 2), and the several-k build (k / 4, k / 2, k in one call against the
+    k build alone). The first two are scans of the masks: bytes moved / time against the HBM peak."""
+    import torch
+
+    from paper_2510_19875_b200 import stream as S
+    from paper_2510_19875_b200 import workloads as wl
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    spec = get_spec(args, 0)
+    w = wl.generate(spec, with_v=False)
+    q, k, _ = w.torch_tensors(dev)
+    kw = dict(block_q=spec.block, block_k=spec.block)
+    peak, peak_kind = hbm_peak()
+
+    def best_ms(fn):
+        best = float("inf")
+        for it in range(args.warmup + args.steps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            torch.cuda.synchronize()
+            if it >= args.warmup:
+                best = min(best, a.elapsed_time(b))
+        return best
+
+    big = S.build_mask(q, k, k_top=spec.k_top, want_scores=True, **kw)
+    small = S.build_mask(q, k, k_top=max(1, spec.k_top // 2), **kw)
+    torch.cuda.synchronize()
+    p = S.make_problem(q, k, k_top=spec.k_top, **kw)
+    n_kb = -(-spec.T // spec.block)
+    rows = spec.n_rows
+    mask_bytes = rows * spec.k_top * 4
+    out = {"workload": spec.name, "T": spec.T, "k_top": spec.k_top, "rows": rows, "hbm_peak_gbs": peak, "peak_kind": peak_kind}
+
+    vert = torch.empty((spec.batch, spec.n_q_heads, n_kb), dtype=torch.float32, device=dev)
+    kurt = torch.empty((spec.batch, spec.n_q_heads), dtype=torch.float32, device=dev)
+    ws = S.new_workspace(p, dev)
+    for name, sc in (("vertical_binary", None), ("vertical_weighted", big.scores)):
+        ms = best_ms(lambda: S.stream_vertical_scores(p, big.mask, sc, vert, kurt, ws, ws.numel()))
+        nbytes = mask_bytes * (2 if sc is not None else 1) + vert.numel() * 4
+        out[name] = {"ms": ms, "bytes": nbytes, "gbs": nbytes / (ms * 1e-3) / 1e9, "frac_of_hbm_peak": nbytes / (ms * 1e-3) / 1e9 / peak}
+
+    diff = torch.empty_like(big.mask)
+    dsc = torch.empty_like(big.scores)
+    ms = best_ms(lambda: S.stream_mask_difference(rows, spec.k_top, big.mask, big.scores, small.mask.shape[-1], small.mask, diff, dsc))
+    nbytes = mask_bytes * 4 + small.mask.numel() * 4  # mask and scores of a in, of the difference out; mask b in
+    out["mask_difference"] = {"ms": ms, "bytes": nbytes, "gbs": nbytes / (ms * 1e-3) / 1e9, "frac_of_hbm_peak": nbytes / (ms * 1e-3) / 1e9 / peak}
+
+    ks = sorted({max(1, spec.k_top // 4), max(1, spec.k_top // 2), spec.k_top})
+    one = best_ms(lambda: S.build_mask(q, k, k_top=spec.k_top, impl=args.kernels, **kw))
+    res = None
+
+    def multi():
+        nonlocal res
+        res = S.build_masks(q, k, ks, impl=args.kernels, **kw)
+    shared = best_ms(multi)
+    out["several_k"] = {"k_list": ks, "ms": shared, "ms_largest_k_alone": one, "ratio": shared / one,
+                        "tiles_scored": int(res.stats().tiles_scored)}
+    print(json.dumps(out))
+
+
 def main():
     args = parse_args()
+    if args.extras:
+        run_extras(args)
+        return
     if args.block_q == 1:
         run_per_token(args)
         return

@@ -482,10 +482,10 @@ __device__ void softmax_role(const Params &P, Tail *tl, unsigned char *p_ptr, un
                 esum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
             };
             auto masked_max = [&]() {
-                float mx = -CUDART_INF_F;
+                float x[64];
 #pragma unroll
-                for (int i = 0; i < 64; ++i) mx = fmaxf(mx, i < n_hi ? __uint_as_float(sr[i]) : -CUDART_INF_F);
-                return mx;
+                for (int i = 0; i < 64; ++i) x[i] = i < n_hi ? __uint_as_float(sr[i]) : -CUDART_INF_F;
+                return max_of_64(x);
             };
             // the token's first allowed logits set its reference (once per pair)
             if (__any_sync(0xffffffffu, ref == -CUDART_INF_F && n_hi > 0)) {

@@ -274,15 +274,11 @@ __device__ void epilogue_role(const Params &P, Tail *tl, unsigned tmem_base, int
                             const long long rem_k = g.T - (long long)blk * kBlk;
                             int lo = (g.causal && blk == qb) ? key : 0;
                             if (key >= rem_k) lo = kBlk;  // key beyond T
-                            float best = -CUDART_INF_F;
-                            if (lo == 0 && m_lim == kBlk) {
+                            if (lo != 0 || m_lim != kBlk) {  // the diagonal block, or a block across T
 #pragma unroll
-                                for (int i = 0; i < 64; ++i) best = fmaxf(best, v[i]);
-                            } else {
-#pragma unroll
-                                for (int i = 0; i < 64; ++i)
-                                    if (i >= lo && i < m_lim) best = fmaxf(best, v[i]);
+                                for (int i = 0; i < 64; ++i) v[i] = (i >= lo && i < m_lim) ? v[i] : -CUDART_INF_F;
                             }
+                            float best = max_of_64(v);
                             best = warp_max(best);
                             if (lane == 0) tl->part[r][c][wq & 1] = best;
                         }

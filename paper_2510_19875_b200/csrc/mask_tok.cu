@@ -245,15 +245,11 @@ mask_tok_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                             long long lim = g.T - k0;
                             if (g.causal) lim = min(lim, e_tq - k0 + 1);
                             const int n_hi = (int)max(0ll, min(lim, (long long)kBlk));
-                            float best = -CUDART_INF_F;
-                            if (n_hi == kBlk) {
+                            if (n_hi != kBlk) {  // the token's own block, or a block across T
 #pragma unroll
-                                for (int j = 0; j < 64; ++j) best = fmaxf(best, v[j]);
-                            } else {
-#pragma unroll
-                                for (int j = 0; j < 64; ++j)
-                                    if (j < n_hi) best = fmaxf(best, v[j]);
+                                for (int j = 0; j < 64; ++j) v[j] = j < n_hi ? v[j] : -CUDART_INF_F;
                             }
+                            const float best = max_of_64(v);
                             if (pos >= 0) scores[pos * kPad + epi_tok] = best;
                         }
                     }

@@ -299,8 +299,9 @@ stream_status stream_selftest_bounded_wait(int64_t limit_cycles, void *workspace
                                            void *cuda_stream);
 
 /*
- * Bytes of device staging stream_run_host needs: room for Q, K, V, the mask, the output and the
- * mask workspace, each 256-byte aligned. 0 if the problem is invalid or unsupported.
+ * Bytes of device staging stream_run_host and stream_run_host_var need: room for Q, K, V, the mask,
+ * the output, the mask workspace and one k per query block, each 256-byte aligned. 0 if the problem
+ * is invalid or unsupported.
  */
 size_t stream_host_staging_bytes(const stream_problem *p);
 
@@ -324,6 +325,19 @@ size_t stream_host_staging_bytes(const stream_problem *p);
 stream_status stream_run_host(const stream_problem *p, const void *q_host, const void *k_host, const void *v_host,
                               int32_t *mask_host, void *out_host, float scale, void *staging,
                               size_t staging_bytes, void *cuda_stream);
+
+/*
+ * stream_run_host with a sparsity constant of its own for every query block (the variable-k build
+ * of stream_build_mask_var, Section 4.2's remedy for the harder pruning of late rows, followed by
+ * the sparse attention on its masks), from HOST memory and pipelined the same way.
+ *
+ *   k_row_host   HOST int32 [ceil(T/block_q)], e.g. from stream_k_schedule; entries outside
+ *                1 .. k_top are clamped. It is copied to the staging buffer ahead of the first chunk.
+ * Everything else as stream_run_host (same staging size).
+ */
+stream_status stream_run_host_var(const stream_problem *p, const void *q_host, const void *k_host, const void *v_host,
+                                  const int32_t *k_row_host, int32_t *mask_host, void *out_host, float scale, void *staging,
+                                  size_t staging_bytes, void *cuda_stream);
 
 #ifdef __cplusplus
 }

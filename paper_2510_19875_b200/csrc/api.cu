@@ -73,7 +73,7 @@ stream_status make_geom(const stream_problem *p, Geom *g) {
 
 size_t elem_size(int dtype) { return dtype == STREAM_F32 ? 4 : 2; }
 
-struct StagingLayout { size_t q, k, v, mask, out, ws, total; };
+struct StagingLayout { size_t q, k, v, mask, out, ws, k_row, total; };
 
 StagingLayout staging_layout(const stream_problem *p, const Geom &g) {
     StagingLayout s;
@@ -81,7 +81,9 @@ StagingLayout staging_layout(const stream_problem *p, const Geom &g) {
     size_t qb = (size_t)g.batch * g.H * g.T * g.d * e, kb = (size_t)g.batch * g.G * g.T * g.d * e;
     size_t mb = (size_t)g.batch * g.H * g.n_qb * g.k_top * sizeof(int32_t);
     s.q = 0; s.k = s.q + align256(qb); s.v = s.k + align256(kb); s.mask = s.v + align256(kb);
-    s.out = s.mask + align256(mb); s.ws = s.out + align256(qb); s.total = s.ws + sizeof(WorkspaceHeader);
+    s.out = s.mask + align256(mb); s.ws = s.out + align256(qb);
+    s.k_row = s.ws + sizeof(WorkspaceHeader);  // one k per query block, for the variable-k path
+    s.total = s.k_row + align256((size_t)g.n_qb * sizeof(int32_t));
     return s;
 }
 
@@ -354,9 +356,10 @@ size_t stream_host_staging_bytes(const stream_problem *p) {
     return staging_layout(p, g).total;
 }
 
-stream_status stream_run_host(const stream_problem *p, const void *q_host, const void *k_host, const void *v_host,
-                              int32_t *mask_host, void *out_host, float scale, void *staging,
-                              size_t staging_bytes, void *cuda_stream) {
+// Both host entry points: k_row_host == NULL is the fixed-k path.
+static stream_status run_host_impl(const stream_problem *p, const void *q_host, const void *k_host, const void *v_host,
+                                   const int32_t *k_row_host, int32_t *mask_host, void *out_host, float scale, void *staging,
+                                   size_t staging_bytes, void *cuda_stream) {
     Geom g;
     stream_status rc = make_geom(p, &g);
     if (rc != STREAM_OK) return rc;
@@ -385,6 +388,11 @@ stream_status stream_run_host(const stream_problem *p, const void *q_host, const
     STREAM_TRY(cudaEventRecord(hp->start, st), "cudaEventRecord");
     STREAM_TRY(cudaStreamWaitEvent(hp->in, hp->start, 0), "cudaStreamWaitEvent");
     STREAM_TRY(cudaStreamWaitEvent(hp->out, hp->start, 0), "cudaStreamWaitEvent");
+    const int32_t *k_row_dev = nullptr;
+    if (k_row_host != nullptr) {  // ahead of the first chunk on the same stream: in place before its kernels wait on it
+        STREAM_TRY(cudaMemcpyAsync(base + s.k_row, k_row_host, (size_t)g.n_qb * sizeof(int32_t), cudaMemcpyHostToDevice, hp->in), "H2D k_row");
+        k_row_dev = (const int32_t *)(base + s.k_row);
+    }
     const int n_chunks = g.batch * g.G;
     const size_t q_head = (size_t)g.T * g.d * e, m_head = (size_t)g.n_qb * g.k_top * sizeof(int32_t);
     int unit = 0;  // running number of the (chunk, heads) units, for the ring of events
@@ -409,8 +417,8 @@ stream_status stream_run_host(const stream_problem *p, const void *q_host, const
             STREAM_TRY(cudaMemcpyAsync(base + s.q + qo, (const char *)q_host + qo, q_bytes, cudaMemcpyHostToDevice, hp->in), "H2D q");
             STREAM_TRY(cudaEventRecord(in_done, hp->in), "cudaEventRecord");
             STREAM_TRY(cudaStreamWaitEvent(st, in_done, 0), "cudaStreamWaitEvent");
-            rc = stream_build_mask(&sub, base + s.q + qo, base + s.k + ko, (int32_t *)(base + s.mask + mo), nullptr, base + s.ws,
-                                   sizeof(WorkspaceHeader), cuda_stream);
+            rc = build_mask_impl(&sub, base + s.q + qo, base + s.k + ko, k_row_dev, (int32_t *)(base + s.mask + mo), nullptr,
+                                 base + s.ws, sizeof(WorkspaceHeader), cuda_stream);
             if (rc != STREAM_OK) return rc;
             rc = stream_sparse_attention(&sub, base + s.q + qo, base + s.k + ko, base + s.v + ko,
                                          (const int32_t *)(base + s.mask + mo), scale, base + s.out + qo, cuda_stream);
@@ -426,6 +434,19 @@ stream_status stream_run_host(const stream_problem *p, const void *q_host, const
     STREAM_TRY(cudaStreamWaitEvent(st, hp->finish, 0), "cudaStreamWaitEvent");
 #undef STREAM_TRY
     return STREAM_OK;
+}
+
+stream_status stream_run_host(const stream_problem *p, const void *q_host, const void *k_host, const void *v_host,
+                              int32_t *mask_host, void *out_host, float scale, void *staging,
+                              size_t staging_bytes, void *cuda_stream) {
+    return run_host_impl(p, q_host, k_host, v_host, nullptr, mask_host, out_host, scale, staging, staging_bytes, cuda_stream);
+}
+
+stream_status stream_run_host_var(const stream_problem *p, const void *q_host, const void *k_host, const void *v_host,
+                                  const int32_t *k_row_host, int32_t *mask_host, void *out_host, float scale, void *staging,
+                                  size_t staging_bytes, void *cuda_stream) {
+    if (k_row_host == nullptr) { set_error("k_row_host must not be NULL (use stream_run_host for one k)"); return STREAM_ERR_INVALID_ARG; }
+    return run_host_impl(p, q_host, k_host, v_host, k_row_host, mask_host, out_host, scale, staging, staging_bytes, cuda_stream);
 }
 
 }  // extern "C"

@@ -8,7 +8,8 @@
 //     S = [Q_0; Q_1] [K_a; K_b]^T      (128 x 128, fp32 in TMEM)
 // holds row 0's logits in its upper-left quadrant and row 1's in its lower-right one.
 //
-// Two softmax groups of four warps take the entries in turn (entry n belongs to group n % 2), so
+// Two softmax groups of four warps take a pair's entries in turn (its n-th kept entry belongs to
+// group n % 2, so that a pair's arithmetic does not depend on what the CTA did before), so
 // that one group's chain of waits, TMEM loads, exponentials and fences runs beside the other's.
 // A thread owns one query token (TMEM lane) of its group's entries: it reads the token's 64
 // logits, applies the element-level mask C, and writes P = exp2(scale (s - ref)) as bf16 into
@@ -17,10 +18,12 @@
 //     O_g[lanes 0..63]   += P[rows 0..63]   V_a,      O_g[lanes 64..127] += P[rows 64..127] V_b
 // (128 x 128, fp32, accumulated in TMEM per group g; V tiles MN-major), add each row's
 // contribution and leave the other row's lanes alone. `ref` is a per-token reference the group keeps
-// instead of the exact running maximum: it is raised (and the token's O_g lane and sum rescaled
-// in place) only when the maximum has grown by more than a factor 2^8 of exp2's argument, so P
-// stays below 2^8 and rescaling is rare. At the end of a pair the two groups exchange (ref, sum)
-// per token, bring O_0 and O_1 to the common reference, add, normalise and store.
+// instead of the exact running maximum (bf16 P and fp32 sums keep their relative precision
+// whatever the reference, as long as nothing overflows): the maximum of the token's first allowed
+// logits, moved (with the token's O_g lane and sum rescaled in place) only when a logit has
+// outgrown it by about 2^30 in exp2's argument, which the entry's sum of P shows. At the end of a
+// pair the two groups exchange (ref, sum) per token, bring O_0 and O_1 to the common reference,
+// add, normalise and store.
 //
 // Roles (384 threads): warp 0 TMA producer (converged, one elected lane issues; two independent
 // non-blocking load streams, K with Q and V); warp 1 issues the Q K^T chains and owns TMEM; warp 3
@@ -62,7 +65,7 @@ constexpr float kLazySum = 68719476736.f;   // 2^36 = 64 * 2^30: the 64 P of an 
 struct Tail {
     unsigned long long q_full, q_empty;
     unsigned long long k_full[kMaxKStages], k_empty[kMaxKStages], v_full[kMaxVStages], v_empty[kMaxVStages];
-    // Per group g (entries n with n % 2 == g): logits ready / read, P published, product added.
+    // Per group g (a pair's kept entries n with n % 2 == g): logits ready / read, P published, product added.
     // o_full[g] also tells the group that its P buffer is free again.
     unsigned long long s_full[2], s_empty[2], p_full[2], o_full[2];
     unsigned long long m_full[kMaskSlots], m_empty[kMaskSlots];
@@ -292,10 +295,11 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
 // The two issuing roles are run by all 32 lanes of their warps, converged: the waits are
 // warp-wide, one elected lane issues.
 
-// S_g = [Q_0; Q_1] [K_a; K_b]^T for every kept entry (g = entry count % 2, over the whole kernel).
+// S_g = [Q_0; Q_1] [K_a; K_b]^T for every kept entry (g = the entry's number within its pair % 2).
 __device__ void qk_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_smem, unsigned tmem_base) {
     const Geom &g = P.g;
-    Ring ks, sb, ms;
+    Ring ks, ms;
+    unsigned cnt[2] = {0, 0};  // entries each group has had over the whole kernel
     unsigned q_par = 0;
     const unsigned q_lo = desc_lo_sw128(q_smem, 16), k_lo = desc_lo_sw128(k_smem, 16);
     for (int id = blockIdx.x; id < P.n_items; id += gridDim.x) {
@@ -308,9 +312,10 @@ __device__ void qk_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_s
         }
         for (int i = 0; i < n_entries; ++i) {
             if (!wait_w(smem_u32(&tl->k_full[ks.idx]), ks.phase, tl, 202)) return;
-            if (!wait_w(smem_u32(&tl->s_empty[sb.idx]), sb.phase ^ 1, tl, 203)) return;
+            const unsigned gi = (unsigned)(i & 1), use = cnt[gi]++;  // entry i of a pair belongs to group i % 2
+            if (!wait_w(smem_u32(&tl->s_empty[gi]), (use & 1u) ^ 1u, tl, 203)) return;
             tc_fence_after();
-            const unsigned d_tmem = tmem_base + sb.idx * 128;
+            const unsigned d_tmem = tmem_base + gi * 128;
             const unsigned b_lo = k_lo + ks.idx * (kOperand >> 4);
             if (elect_one()) {
 #pragma unroll
@@ -319,12 +324,11 @@ __device__ void qk_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_s
                     for (int k4 = 0; k4 < 4; ++k4)
                         tc_mma_bf16_split(d_tmem, q_lo + ((c * 2 * kHalfTile + k4 * 32) >> 4), kHiK,
                                           b_lo + ((c * 2 * kHalfTile + k4 * 32) >> 4), kHiK, kIdescQK, (c | k4) != 0);
-                tc_commit(smem_u32(&tl->s_full[sb.idx]));
+                tc_commit(smem_u32(&tl->s_full[gi]));
                 tc_commit(smem_u32(&tl->k_empty[ks.idx]));
                 if (i + 1 == n_entries) tc_commit(smem_u32(&tl->q_empty));  // that was the pair's last use of Q
             }
             __syncwarp();
-            sb.advance(2);
             ks.advance(P.n_k_stages);
         }
         if (elect_one()) mbar_arrive(smem_u32(&tl->m_empty[ms.idx]));
@@ -336,7 +340,8 @@ __device__ void qk_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_s
 // O_g (+)= P_g [V_a; V_b] for every kept entry; a group's first entry of a pair starts its O afresh.
 __device__ void pv_role(const Params &P, Tail *tl, unsigned p_smem, unsigned v_smem, unsigned tmem_base) {
     const Geom &g = P.g;
-    Ring gr, vs, ms;  // gr: group = O buffer of the entry; vs: its V stage
+    Ring vs, ms;  // vs: the entry's V stage
+    unsigned cnt[2] = {0, 0};  // entries each group has had over the whole kernel
     // the MN-major V tiles have their two 64-channel halves kHalfTile apart
     const unsigned p_lo = desc_lo_sw128(p_smem, 16), v_lo = desc_lo_sw128(v_smem, kHalfTile);
     for (int id = blockIdx.x; id < P.n_items; id += gridDim.x) {
@@ -346,12 +351,13 @@ __device__ void pv_role(const Params &P, Tail *tl, unsigned p_smem, unsigned v_s
         unsigned fresh = 3u;  // bit g: group g has not added anything for this pair yet
         for (int i = 0; i < n_entries; ++i) {
             if (!wait_w(smem_u32(&tl->v_full[vs.idx]), vs.phase, tl, 205)) return;
-            if (!wait_w(smem_u32(&tl->p_full[gr.idx]), gr.phase, tl, 204)) return;  // also: O_g rescaled if it had to be
+            const unsigned gi = (unsigned)(i & 1), use = cnt[gi]++;  // group = O buffer of the entry
+            if (!wait_w(smem_u32(&tl->p_full[gi]), use & 1u, tl, 204)) return;  // also: O_g rescaled if it had to be
             tc_fence_after();
-            const unsigned d_tmem = tmem_base + 256 + gr.idx * 128;
-            const unsigned a_lo = p_lo + gr.idx * (kPBytes >> 4), b_lo = v_lo + vs.idx * (kOperand >> 4);
-            const unsigned keep = ((fresh >> gr.idx) & 1u) ^ 1u;
-            fresh &= ~(1u << gr.idx);
+            const unsigned d_tmem = tmem_base + 256 + gi * 128;
+            const unsigned a_lo = p_lo + gi * (kPBytes >> 4), b_lo = v_lo + vs.idx * (kOperand >> 4);
+            const unsigned keep = ((fresh >> gi) & 1u) ^ 1u;
+            fresh &= ~(1u << gi);
             if (elect_one()) {
 #pragma unroll
                 for (int tile = 0; tile < 2; ++tile) {  // row `tile` of the pair: its P rows, its V tile, its lanes
@@ -361,11 +367,10 @@ __device__ void pv_role(const Params &P, Tail *tl, unsigned p_smem, unsigned v_s
                         tc_mma_bf16_split_masked(d_tmem, a_lo + ((s4 * 32) >> 4), kHiK, b_lo + ((tile * kTile + s4 * 2048) >> 4),
                                                  kHiK, kIdescPV, s4 != 0 ? 1u : keep, lo_off, lo_off, hi_off, hi_off);
                 }
-                tc_commit(smem_u32(&tl->o_full[gr.idx]));  // product added: the group's P buffer is free
+                tc_commit(smem_u32(&tl->o_full[gi]));  // product added: the group's P buffer is free
                 tc_commit(smem_u32(&tl->v_empty[vs.idx]));
             }
             __syncwarp();
-            gr.advance(2);
             vs.advance(P.n_v_stages);
         }
         if (elect_one()) mbar_arrive(smem_u32(&tl->m_empty[ms.idx]));
@@ -397,7 +402,7 @@ __device__ __forceinline__ void rescale_lane(unsigned taddr, float f) {
 }
 
 // One softmax group: four warps, thread = query token (TMEM lane) `row` of the pair, for the
-// entries n with n % 2 == grp (n counts the kept entries over the whole kernel, as in every role).
+// entries n with n % 2 == grp (n numbers the kept entries of each pair, as in every role).
 // The waits are warp-wide (same answer in every lane), so the warp stays converged for the
 // warp-collective TMEM loads and stores and leaves together if the CTA aborts.
 __device__ void softmax_role(const Params &P, Tail *tl, unsigned char *p_ptr, unsigned tmem_base, int t) {
@@ -415,7 +420,6 @@ __device__ void softmax_role(const Params &P, Tail *tl, unsigned char *p_ptr, un
     const unsigned s_addr = tmem_base + grp * 128 + half * 64 + lane_off;
     const unsigned o_own = tmem_base + 256 + grp * 128 + lane_off, o_other = tmem_base + 256 + (grp ^ 1) * 128 + lane_off;
     unsigned s_par = 0, o_par = 0, x_par = 0;
-    unsigned n = 0;  // kept entries so far
     Ring ms;
     for (int id = blockIdx.x; id < P.n_items; id += gridDim.x) {
         const Item it = decode_item(P, id);
@@ -426,9 +430,10 @@ __device__ void softmax_role(const Params &P, Tail *tl, unsigned char *p_ptr, un
         float ref = -CUDART_INF_F, l = 0.f;
         bool pending = false;  // a P V chain of this group and pair may still be running
         Entry cur;
+        unsigned n = 0;
         for (int e = next_entry(rows, P.row_stride, -1, g.k_top, &cur); e < g.k_top;
              e = next_entry(rows, P.row_stride, e, g.k_top, &cur), ++n) {
-            if ((int)(n & 1u) != grp) continue;
+            if ((int)(n & 1u) != grp) continue;  // n: the entry's number within the pair
             // the token's 64 logits against its row's key block
             if (!wait_w(s_full, s_par, tl, 301)) return;
             s_par ^= 1;

@@ -102,6 +102,8 @@ def _load():
     lib.stream_host_staging_bytes.argtypes = [P]
     lib.stream_run_host.restype = ctypes.c_int
     lib.stream_run_host.argtypes = [P, vp, vp, vp, vp, vp, ctypes.c_float, vp, sz, vp]
+    lib.stream_run_host_var.restype = ctypes.c_int
+    lib.stream_run_host_var.argtypes = [P, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, sz, vp]
     _lib = lib
     return lib
 
@@ -223,6 +225,14 @@ def stream_run_host(p: StreamProblem, q_host, k_host, v_host, mask_host, out_hos
                     staging_bytes: int, stream=None) -> None:
     _raise(_load().stream_run_host(ctypes.byref(p), _addr(q_host), _addr(k_host), _addr(v_host), _addr(mask_host),
                                    _addr(out_host), float(scale), _addr(staging), staging_bytes, _stream_handle(stream)))
+
+
+def stream_run_host_var(p: StreamProblem, q_host, k_host, v_host, k_row_host, mask_host, out_host, scale: float, staging,
+                        staging_bytes: int, stream=None) -> None:
+    """The host path with one k per query block (``k_row_host``: HOST int32 array)."""
+    _raise(_load().stream_run_host_var(ctypes.byref(p), _addr(q_host), _addr(k_host), _addr(v_host), _addr(k_row_host),
+                                       _addr(mask_host), _addr(out_host), float(scale), _addr(staging), staging_bytes,
+                                       _stream_handle(stream)))
 
 
 # ----------------------------------------------------------------------------------------------
@@ -347,12 +357,18 @@ def sparse_attention(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, mask: to
 
 def run_host(q_host: torch.Tensor, k_host: torch.Tensor, v_host: torch.Tensor, mask_host: torch.Tensor,
              out_host: torch.Tensor, staging: torch.Tensor, *, block_q: int, block_k: int, k_top: int,
-             causal: bool = True, scale: float = 0.0, impl: str = "auto", stream=None) -> None:
-    """Whole path from (pinned) host tensors through a caller-provided device staging buffer."""
+             causal: bool = True, scale: float = 0.0, impl: str = "auto", k_row: torch.Tensor | None = None, stream=None) -> None:
+    """Whole path from (pinned) host tensors through a caller-provided device staging buffer. With
+    ``k_row`` (HOST int32 tensor, one k per query block) the mask is the variable-k build."""
     if q_host.is_cuda or not staging.is_cuda:
         raise ValueError("q/k/v/mask/out live on the host, staging on the device")
     p = make_problem(q_host, k_host, block_q=block_q, block_k=block_k, k_top=k_top, causal=causal, impl=impl)
-    stream_run_host(p, q_host, k_host, v_host, mask_host, out_host, scale, staging, staging.numel(), stream)
+    if k_row is None:
+        stream_run_host(p, q_host, k_host, v_host, mask_host, out_host, scale, staging, staging.numel(), stream)
+    else:
+        if k_row.is_cuda or k_row.dtype != torch.int32 or not k_row.is_contiguous() or k_row.numel() != n_query_blocks(p):
+            raise ValueError("k_row must be a contiguous int32 HOST tensor with one entry per query block")
+        stream_run_host_var(p, q_host, k_host, v_host, k_row, mask_host, out_host, scale, staging, staging.numel(), stream)
 
 
 def vertical_scores(p: StreamProblem, mask: torch.Tensor, scores: torch.Tensor | None = None, stream=None):

@@ -100,6 +100,13 @@ def test_cpu_tensors_are_refused(S):
         S.sparse_attention(q, q, q, torch.zeros(1, 1, 2, 2, dtype=torch.int32), block_q=32, block_k=32)
 
 
+def test_run_host_var_needs_a_schedule(S):
+    p = good_problem(S)
+    with pytest.raises(S.StreamError) as e:
+        S.stream_run_host_var(p, 256, 256, 256, None, 256, 256, 0.0, 256, 1 << 30, stream=0)
+    assert e.value.status == S.STREAM_ERR_INVALID_ARG
+
+
 def test_staging_size_covers_all_buffers(S):
     p = good_problem(S)
     e = 2

@@ -321,6 +321,26 @@ def test_run_host_matches_device_calls(S):
     assert torch.equal(out_host, out_ref.cpu())
 
 
+def test_run_host_var_matches_device_calls(S):
+    """The host path with one k per query block against the device calls it is made of."""
+    w = wl.generate(small_spec(dtype="bf16", d=128, block=64, T=4096, k_top=8, n_q_heads=8, n_kv_heads=2, sink=True, batch=2))
+    qh, kh, vh = w.torch_tensors("cpu", pin=True)
+    q, k, v = qh.cuda(), kh.cuda(), vh.cuda()
+    p = S.make_problem(qh, kh, block_q=64, block_k=64, k_top=8)
+    k_row = S.k_schedule(p, 0.1)
+    assert k_row.min() < k_row.max()
+    ref = S.build_mask(q, k, block_q=64, block_k=64, k_top=8, k_row=k_row.cuda())
+    out_ref = S.sparse_attention(q, k, v, ref.mask, block_q=64, block_k=64)
+    staging = torch.empty(S.stream_host_staging_bytes(p), dtype=torch.uint8, device="cuda")
+    mask_host = torch.empty(ref.mask.shape, dtype=torch.int32).pin_memory()
+    out_host = torch.empty(out_ref.shape, dtype=out_ref.dtype).pin_memory()
+    S.run_host(qh, kh, vh, mask_host, out_host, staging, block_q=64, block_k=64, k_top=8, k_row=k_row)
+    torch.cuda.synchronize()
+    assert torch.equal(mask_host, ref.mask.cpu())
+    assert torch.equal(out_host, out_ref.cpu())
+    assert ((mask_host >= 0).sum(-1)[0, 0] == torch.minimum(k_row, torch.arange(1, k_row.numel() + 1, dtype=torch.int32))).all()
+
+
 @pytest.mark.parametrize("kw", [dict(), dict(T=5000, k_top=5, n_q_heads=7, n_kv_heads=1), dict(T=3000, k_top=3, n_q_heads=6, n_kv_heads=2, batch=2)])
 def test_vertical_scores_and_kurtosis(S, kw):
     """Column sums of the GPU mask (binary and score-weighted) and their kurtosis against the oracle

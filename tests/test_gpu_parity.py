@@ -173,6 +173,35 @@ def test_mask_per_token_tensor_core_repeats_and_matches_generic(S):
     assert st.tile_products >= st.tiles_scored // 64              # every needed tile is inside a computed product
 
 
+def test_mask_per_token_strided_inputs_and_limits(S):
+    """[B, T, H, d] storage through [B, H, T, d] strides gives the same per-token mask (the kernel
+    reads Q rows straight from global memory with the caller's strides); shapes the per-token
+    tensor-core kernel does not take are refused when it is asked for by name and run on the
+    generic kernel otherwise."""
+    w = wl.generate(tc_spec(T=1500, k_top=4, n_q_heads=4, n_kv_heads=2))
+    q, k, _ = w.torch_tensors("cuda")
+    ref = S.build_mask(q, k, block_q=1, block_k=64, k_top=4, impl="tensor")
+    assert ref.stats().tile_products > 0
+    qs = q.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    ks = k.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    assert not qs.is_contiguous()
+    got = S.build_mask(qs, ks, block_q=1, block_k=64, k_top=4, impl="tensor")
+    assert torch.equal(got.mask, ref.mask)
+    # one k per call only: the variable-k build for per-token rows is the generic kernel's
+    p = S.make_problem(q, k, block_q=1, block_k=64, k_top=4, impl="tensor")
+    k_row = torch.full((1500,), 3, dtype=torch.int32, device="cuda")
+    ws = S.new_workspace(p, q.device)
+    with pytest.raises(S.StreamError) as e:
+        S.stream_build_mask_var(p, q, k, k_row, ref.mask.clone(), None, ws, ws.numel())
+    assert e.value.status == S.STREAM_ERR_UNSUPPORTED
+    var = S.build_mask(q, k, block_q=1, block_k=64, k_top=4, k_row=k_row)   # impl auto: generic kernel
+    assert var.stats().tile_products == 0 and ((var.mask >= 0).sum(-1) <= 3).all()
+    # block_k other than 64 is not the tensor-core kernel's either
+    with pytest.raises(S.StreamError) as e:
+        S.build_mask(q, k, block_q=1, block_k=32, k_top=4, impl="tensor")
+    assert e.value.status == S.STREAM_ERR_UNSUPPORTED
+
+
 def test_mask_generic_non_causal(S):
     w = wl.generate(small_spec(T=900, k_top=6, n_q_heads=2, n_kv_heads=2))
     assert_mask_parity(S, w, None, impl="generic", score_cache=False, causal=False)

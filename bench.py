@@ -479,6 +479,33 @@ def run_ours(args):
         rows = sweep_rows(wl.SWEEP_T[:3], dev)
         line["sweep"] = {"rows": [{k2: r[k2] for k2 in ("T", "levels", "mask_ms", "attention_ms", "peak_device_bytes")} for r in rows],
                          **sweep_fits(rows)}
+        # and the two small workloads (a single fp32 head; a 16k-token GQA layer), device-resident, best of 3
+        small = {}
+        for name in ("single_head_fp32", "gqa_layer_16k"):
+            if name == spec.name:
+                continue
+            sp = wl.SPECS[name]
+            ws_ = wl.generate(sp)
+            q2, k2, v2 = ws_.torch_tensors(dev)
+            p2 = S.make_problem(q2, k2, block_q=sp.block, block_k=sp.block, k_top=sp.k_top, impl=args.kernels)
+            m2 = torch.empty((sp.batch, sp.n_q_heads, S.n_query_blocks(p2), sp.k_top), dtype=torch.int32, device=dev)
+            o2 = torch.empty_like(q2)
+            w2 = S.new_workspace(p2, dev)
+            best = [float("inf"), float("inf")]
+            for it in range(5):
+                e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+                e0.record()
+                S.stream_build_mask(p2, q2, k2, m2, None, w2, w2.numel(), stream)
+                e1.record()
+                S.stream_sparse_attention(p2, q2, k2, v2, m2, 0.0, o2, stream)
+                e2.record()
+                torch.cuda.synchronize()
+                if it >= 2:
+                    best = [min(best[0], e0.elapsed_time(e1)), min(best[1], e1.elapsed_time(e2))]
+            small[name] = {"mask_ms": best[0], "attention_ms": best[1], "T": sp.T, "dtype": sp.dtype,
+                           "value": sp.batch * sp.n_q_heads * sp.T / ((best[0] + best[1]) * 1e-3), "unit": UNIT}
+            del q2, k2, v2, m2, o2
+        line["other_workloads"] = small
     if not args.no_cpu_baseline:
         rate, threads, sample = oracle_sample_rate(spec, w, args.cpu_seconds)
         line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample}

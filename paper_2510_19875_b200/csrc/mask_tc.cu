@@ -41,7 +41,8 @@ constexpr int kHalfTile = kBlk * 128;          // 64 rows x 128 bytes (one 64-ch
 constexpr int kStageBytes = 4 * kHalfTile;     // [2 channel halves][2 tiles]
 constexpr int kQBytes = 2 * kR * kHalfTile;    // [2 channel halves][kR rows]
 constexpr int kMaxJobs = 64;
-constexpr int kListReaders = 1 + kMmaWarps + 4 * kEpiGroups;  // producer warp, MMA warps, epilogue warps
+constexpr int kProducers = 2;     // warps 0 and 14: producer p fills the stage buffers b with b % 2 == p
+constexpr int kListReaders = kProducers + kMmaWarps + 4 * kEpiGroups;  // producer, MMA and epilogue warps
 // A parity wait only means something to a thread that saw the phase before it complete, and an
 // arrival only if it cannot come a phase early. So every stage buffer and every TMEM slot
 // belongs to one issuing warp: stage s of the kernel's whole sequence goes, with all its chains,
@@ -113,7 +114,7 @@ __device__ __forceinline__ unsigned long long cache_pack(unsigned tag, float s) 
 // Run by all 32 lanes of warp 0, converged (warp-wide waits, one elected lane issues): a single
 // diverged lane issues TMA copies several times more slowly.
 __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUtensorMap *tk, Tail *tl, unsigned q_smem,
-                              unsigned k_smem) {
+                              unsigned k_smem, int which) {
     Ring st;
     unsigned grp_par = 0, jr_par[kR] = {0, 0, 0, 0};
     for (;;) {
@@ -123,7 +124,7 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
         const int b = tl->grp_b, kvh = tl->grp_kvh, qb = tl->grp_qb, h0 = tl->grp_h0, R = tl->grp_R;
         const int levels = tl->grp_levels;
         // Q tiles of the group's rows (previous group's MMAs are all complete by now)
-        if (tl->grp_new_q && elect_one()) {
+        if (which == 0 && tl->grp_new_q && elect_one()) {
             mbar_arrive_expect_tx(smem_u32(&tl->q_full), (unsigned)(R * 2 * kHalfTile));
             for (int r = 0; r < R; ++r)
                 for (int c = 0; c < 2; ++c)
@@ -140,6 +141,7 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
                 }
                 const int n = tl->n_jobs[li];
                 for (int j = 0; j < n; j += 2) {
+                    if ((st.idx & (kProducers - 1)) != which) { st.advance(kStages); continue; }  // the other producer's buffer
                     if (!mbar_wait_w(smem_u32(&tl->empty[st.idx]), st.phase ^ 1, tl, P.ws, 103)) return;
                     const int two = (j + 1 < n);
                     const int blk0 = tl->jobs_blk[li][j], blk1 = two ? tl->jobs_blk[li][j + 1] : 0;
@@ -168,11 +170,23 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
 // times longer than the tensor core needs for a chain, so one issuing warp would leave it idle
 // most of the time. All issuing warps walk the same unit order; each is run by all 32 lanes,
 // converged: warp-wide waits, one elected lane issues.
+//
+// Which of the owner's two TMEM slots a chain lands in is a fixed function of its place in the
+// unit order, so that the issuing warp and the epilogue groups agree on it without counting each
+// other's chains: on the first level chain r of a stage goes to slot r % 2, later (one chain per
+// stage) the chain of stage s goes to slot (s / kMmaWarps) % 2. Both sides keep one phase bit per
+// slot they use.
+__device__ __forceinline__ int chain_slot(int level, int r, unsigned stage) {
+    return level == 0 ? (r & 1) : (int)((stage / kMmaWarps) & 1u);
+}
+
 __device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_smem, unsigned tmem_base, int which) {
     unsigned grp_par = 0, q_par = 0, jr_par[kR] = {0, 0, 0, 0};
     unsigned stage_seq = 0;   // stages so far, over the whole kernel (the same in every role)
-    unsigned my_chains = 0;   // chains this warp has issued
+    unsigned slot_par = 0;    // bit i: phase of the next use of this warp's slot i
     const unsigned q_lo = desc_lo_sw128(q_smem, 16);
+    const int sidx = which;   // this warp's stage buffer: stage s lands in buffer s % kStages
+    const unsigned a_lo = desc_lo_sw128(k_smem + sidx * kStageBytes, 16);
     for (;;) {
         if (!mbar_wait_w(smem_u32(&tl->jobs_ready[kR]), grp_par, tl, P.ws, 201)) return;
         grp_par ^= 1;
@@ -190,19 +204,20 @@ __device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_
                     if (!mbar_wait_w(smem_u32(&tl->jobs_ready[x]), jr_par[x], tl, P.ws, 203)) return;
                     jr_par[x] ^= 1;
                 }
-                const int n = tl->n_jobs[li];
+                const unsigned n_st = (unsigned)(tl->n_jobs[li] + 1) >> 1;  // stages of this list
                 __syncwarp();
                 if (elect_one()) mbar_arrive(smem_u32(&tl->jobs_ack[li]));  // the count is all this role reads
                 __syncwarp();
                 const int r0 = level == 0 ? 0 : x, r1 = level == 0 ? R : x + 1;
-                for (int j = 0; j < n; j += 2, ++stage_seq) {
-                    if ((int)(stage_seq % kMmaWarps) != which) continue;  // another warp's stage: nothing to do
-                    const int sidx = which;  // = stage_seq % kStages
-                    if (!mbar_wait_w(smem_u32(&tl->full[sidx]), (stage_seq / kStages) & 1u, tl, P.ws, 204)) return;
-                    const unsigned a_lo = desc_lo_sw128(k_smem + sidx * kStageBytes, 16);
-                    for (int r = r0; r < r1; ++r, ++my_chains) {
-                        const int slot = 2 * which + (int)(my_chains & 1u);
-                        if (!mbar_wait_w(smem_u32(&tl->tmem_empty[slot]), ((my_chains >> 1) & 1u) ^ 1u, tl, P.ws, 205)) return;
+                const unsigned s_end = stage_seq + n_st;
+                // this warp's stages of the list: s = which (mod kMmaWarps)
+                for (unsigned s = stage_seq + (((unsigned)which - stage_seq) & (kMmaWarps - 1)); s < s_end; s += kMmaWarps) {
+                    if (!mbar_wait_w(smem_u32(&tl->full[sidx]), (s / kStages) & 1u, tl, P.ws, 204)) return;
+                    for (int r = r0; r < r1; ++r) {
+                        const int sl = chain_slot(level, r, s);
+                        const int slot = 2 * which + sl;
+                        if (!mbar_wait_w(smem_u32(&tl->tmem_empty[slot]), ((slot_par >> sl) & 1u) ^ 1u, tl, P.ws, 205)) return;
+                        slot_par ^= 1u << sl;
                         tc_fence_after();
                         const unsigned d_tmem = tmem_base + slot * 64;
                         const unsigned b_lo = q_lo + r * (kHalfTile >> 4);
@@ -221,21 +236,25 @@ __device__ void mma_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_
                         __syncwarp();
                     }
                 }
+                stage_seq = s_end;
             }
         }
     }
 }
 
-// One epilogue group (four warps, one per TMEM lane quarter). Both groups walk every chain of
-// every list, but group `grp` only waits for and reduces those in slot `grp` of the issuing
-// warp's two: a slot's barriers are then used by one group only, which sees every phase of them.
+// One epilogue group (four warps, one per TMEM lane quarter). Group `grp` waits for and reduces
+// the chains that land in slot `grp` of their issuing warp (chain_slot): a slot's barriers are
+// then used by one group only, which sees every phase of them. It steps over the other group's
+// chains without looking at them: the bookkeeping of a warp is serial code, and what it spends
+// there it cannot spend reducing.
 __device__ void epilogue_role(const Params &P, Tail *tl, unsigned tmem_base, int wq, int grp, int lane) {
     const Geom &g = P.g;
     unsigned grp_par = 0, jr_par[kR] = {0, 0, 0, 0};
     unsigned stage_seq = 0;
-    unsigned chains = 0;  // chains each issuing warp has produced so far, mod 4: two bits per warp
+    unsigned full_par = 0;  // bit w: phase of the next use of issuing warp w's slot `grp`
     const int tile = wq >> 1;                // which tile of the pair this warp's lanes hold
     const int key = (wq & 1) * 32 + lane;    // key index inside the tile
+    const unsigned t_lane = tmem_base + ((unsigned)(wq * 32) << 16) + grp * 64;
     for (;;) {
         if (!mbar_wait(smem_u32(&tl->jobs_ready[kR]), grp_par, tl, P.ws, 301)) return;
         grp_par ^= 1;
@@ -243,6 +262,36 @@ __device__ void epilogue_role(const Params &P, Tail *tl, unsigned tmem_base, int
         const int R = tl->grp_R, qb = tl->grp_qb, levels = tl->grp_levels;
         const long long rem_q = g.T - (long long)qb * kBlk;
         const int m_lim = rem_q < kBlk ? (int)rem_q : kBlk;  // query tokens of this block inside T
+        // One chain of this group: stage s, row r, this warp's tile at position c of list li.
+        auto reduce = [&](unsigned s, int r, int li, int c, int n) -> bool {
+            const unsigned owner = s & (kMmaWarps - 1);
+            const unsigned slot = 2 * owner + grp;
+            if (!mbar_wait(smem_u32(&tl->tmem_full[slot]), (full_par >> owner) & 1u, tl, P.ws, 303)) return false;
+            full_par ^= 1u << owner;
+            tc_fence_after();
+            if (c < n) {
+                const int blk = tl->jobs_blk[li][c];
+                float v[64];
+                const unsigned taddr = t_lane + owner * 128;
+                tmem_ld_32x32(taddr, v);
+                tmem_ld_32x32(taddr + 32, v + 32);
+                // allowed queries for this key: inside T, and not before the key if causal
+                const long long rem_k = g.T - (long long)blk * kBlk;
+                int lo = (g.causal && blk == qb) ? key : 0;
+                if (key >= rem_k) lo = kBlk;  // key beyond T
+                if (lo != 0 || m_lim != kBlk) {  // the diagonal block, or a block across T
+#pragma unroll
+                    for (int i = 0; i < 64; ++i) v[i] = (i >= lo && i < m_lim) ? v[i] : -CUDART_INF_F;
+                }
+                float best = max_of_64(v);
+                best = warp_max(best);
+                if (lane == 0) tl->part[r][c][wq & 1] = best;
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&tl->tmem_empty[slot]));
+            return true;
+        };
         for (int level = 0; level < levels; ++level) {
             const int lists = level == 0 ? 1 : R;
             for (int x = 0; x < lists; ++x) {
@@ -252,41 +301,24 @@ __device__ void epilogue_role(const Params &P, Tail *tl, unsigned tmem_base, int
                     jr_par[x] ^= 1;
                 }
                 const int n = tl->n_jobs[li];
-                for (int j = 0; j < n; j += 2, ++stage_seq) {
-                    const int c = j + tile;
-                    const int blk = c < n ? tl->jobs_blk[li][c] : -1;
-                    const int r0 = level == 0 ? 0 : x, r1 = level == 0 ? R : x + 1;
-                    const int owner = (int)(stage_seq % kMmaWarps);
-                    for (int r = r0; r < r1; ++r) {
-                        // the owner's chains alternate between its two slots
-                        const unsigned cnt = (chains >> (2 * owner)) & 3u;
-                        const int slot = 2 * owner + (int)(cnt & 1u);
-                        chains = (chains & ~(3u << (2 * owner))) | (((cnt + 1u) & 3u) << (2 * owner));
-                        if ((int)(cnt & 1u) != grp) continue;  // the other group's chain
-                        if (!mbar_wait(smem_u32(&tl->tmem_full[slot]), cnt >> 1, tl, P.ws, 303)) return;
-                        tc_fence_after();
-                        if (blk >= 0) {
-                            const unsigned taddr = tmem_base + slot * 64 + ((unsigned)(wq * 32) << 16);
-                            float v[64];
-                            tmem_ld_32x32(taddr, v);
-                            tmem_ld_32x32(taddr + 32, v + 32);
-                            // allowed queries for this key: inside T, and not before the key if causal
-                            const long long rem_k = g.T - (long long)blk * kBlk;
-                            int lo = (g.causal && blk == qb) ? key : 0;
-                            if (key >= rem_k) lo = kBlk;  // key beyond T
-                            if (lo != 0 || m_lim != kBlk) {  // the diagonal block, or a block across T
-#pragma unroll
-                                for (int i = 0; i < 64; ++i) v[i] = (i >= lo && i < m_lim) ? v[i] : -CUDART_INF_F;
-                            }
-                            float best = max_of_64(v);
-                            best = warp_max(best);
-                            if (lane == 0) tl->part[r][c][wq & 1] = best;
-                        }
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(smem_u32(&tl->tmem_empty[slot]));
+                const unsigned s_end = stage_seq + ((unsigned)(n + 1) >> 1);
+                if (level == 0) {
+                    // every stage serves all rows; rows grp, grp + 2 are this group's
+                    for (unsigned s = stage_seq; s < s_end; ++s) {
+                        const int c = 2 * (int)(s - stage_seq) + tile;
+                        for (int r = grp; r < R; r += 2)
+                            if (!reduce(s, r, li, c, n)) return;
+                    }
+                } else {
+                    // one chain per stage; this group's are the stages with (s / kMmaWarps) % 2 == grp
+                    unsigned s = stage_seq;
+                    while (s < s_end) {
+                        if ((int)((s / kMmaWarps) & 1u) != grp) { s = (s | (kMmaWarps - 1)) + 1; continue; }
+                        if (!reduce(s, x, li, 2 * (int)(s - stage_seq) + tile, n)) return;
+                        ++s;
                     }
                 }
+                stage_seq = s_end;
                 // this list is done for rows r0..r1: tell the controller
                 if (lane == 0) {
                     const int r0 = level == 0 ? 0 : x, r1 = level == 0 ? R : x + 1;
@@ -489,8 +521,8 @@ mask_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     tc_fence_after();
     const unsigned tmem_base = tl->tmem_base;
 
-    if (warp == 0) {
-        producer_role(P, &tmap_q, &tmap_k, tl, q_smem, k_smem);
+    if (warp == 0 || warp == 14) {
+        producer_role(P, &tmap_q, &tmap_k, tl, q_smem, k_smem, warp == 0 ? 0 : 1);
     } else if (warp == 1) {
         mma_role(P, tl, q_smem, k_smem, tmem_base, 0);
     } else if (warp == 2) {

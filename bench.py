@@ -180,15 +180,11 @@ def ncu_traffic(kernel: str, spec):
         return None
 
 
-# Shared-memory traffic per unit of work in the tensor-core kernels' present formulation (bytes that
-# cross the SM's 128-byte-per-clock shared-memory port): what the TMA copies write plus what the
-# tcgen05.mma instructions read as operands.
-#   mask build, per scored tile: the key tile written once (16 KB; shared by the rows of a group at
-#     the first level, counted in full here) + read once as the A operand (16 KB) + the query tile
-#     read as the B operand (8 KB per tile of a two-tile chain)
-#   attention, per kept block: K and V tiles written (32 KB), K and V read as operands (32 KB), the
-#     Q operand (8 KB per block of a two-block chain), P written and read (8 KB + 8 KB)
-SMEM_PORT_BYTES = {"mask_tc_kernel": 40 * 1024, "attn_tc_kernel": 88 * 1024}
+# The two SM units the tensor-core kernels lean on, measured on the device by the library's own
+# probe (stream_probe_unit_rates) right before the timed steps: the bytes per clock one SM's TMA
+# unit brings from L2 into shared memory, and the clocks one tcgen05.mma of the mask kernel's
+# shape takes. The bench line sets each kernel's traffic and instruction count against them.
+TC_KERNELS = ("mask_tc_kernel", "attn_tc_kernel")
 
 
 def rank_env():
@@ -321,6 +317,10 @@ def run_ours(args):
         build_mask()
         S.stream_sparse_attention(p, q, k, v, mask, 0.0, out, stream)
 
+    # the device's own unit rates (two short probe kernels, outside the timed region)
+    unit_rates = None
+    if rank == 0 and spec.dtype == "bf16" and args.kernels != "generic":
+        unit_rates = S.probe_unit_rates(dev, stream)
     for _ in range(args.warmup):
         step()
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
@@ -449,13 +449,23 @@ def run_ours(args):
                             "frac_of_8TBs_nominal": dom["algorithmic_gbs"] / 8000.0,
                             "note": "served by L2: DRAM carries only `traffic`"},
     })
-    if dom["kernel"] in SMEM_PORT_BYTES:
-        work = S_tiles if dominant == "stream_build_mask" else kept
-        port_bytes = work * SMEM_PORT_BYTES[dom["kernel"]]
-        port_peak = 128.0 * n_sm * sm_mhz * 1e6 / 1e9  # GB/s at the sampled SM clock
-        roof["smem_port"] = {"model_bytes": port_bytes, "achieved": port_bytes / (dom["ms"] * 1e-3) / 1e9, "peak": port_peak,
-                             "unit": "GB/s", "frac": port_bytes / (dom["ms"] * 1e-3) / 1e9 / port_peak,
-                             "peak_kind": f"128 B/clk x {n_sm} SMs x {sm_mhz:.0f} MHz (sampled)"}
+    if dom["kernel"] in TC_KERNELS and unit_rates is not None:
+        cycles = dom["ms"] * 1e-3 * sm_mhz * 1e6  # per SM, at the sampled clock
+        if dominant == "stream_build_mask":
+            gathered = int(stats.tiles_fetched) * tile_bytes          # counted by the kernel
+            mma_cycles = S_tiles / 2 * 8 * unit_rates.mma_cycles_m128n64 / n_sm   # chains of two tiles, eight MMAs each
+        else:
+            gathered = kept * 2 * tile_bytes + units * spec.d * esz   # K and V tile per kept block, Q once
+            mma_cycles = None
+        per_clk = gathered / n_sm / cycles
+        roof["unit_rates"] = {
+            "sm_mhz": sm_mhz, "kind": "measured by stream_probe_unit_rates on this device before the timed steps",
+            "tma_bytes_per_clk_per_sm": unit_rates.tma_bytes_per_clk, "mma_m128n64k16_cycles": unit_rates.mma_cycles_m128n64,
+            "tma_gather": {"bytes": gathered, "achieved": per_clk, "peak": unit_rates.tma_bytes_per_clk,
+                           "unit": "B/clk/SM", "frac": per_clk / unit_rates.tma_bytes_per_clk},
+        }
+        if mma_cycles is not None:
+            roof["unit_rates"]["mma_issue"] = {"cycles_needed": mma_cycles, "cycles_measured": cycles, "frac": mma_cycles / cycles}
     line = {
         "metric": METRIC, "value": job_value(world, units, args.steps, total_ms), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,

@@ -81,6 +81,9 @@ typedef struct {
                                multiplies every fetched key tile with 128 tokens at once, so this
                                exceeds tiles_scored / 64); 0 from the other kernels, whose products
                                are exactly the tiles scored */
+    uint64_t tiles_fetched; /* key and query tiles (block x d) the tensor-core block kernel copied into
+                               shared memory: fewer than tiles_scored where a fetched key tile serves
+                               several rows; 0 from the kernels that do not count them */
 } stream_stats;
 
 /* Library version: major * 10000 + minor * 100 + patch. */
@@ -297,6 +300,32 @@ stream_status stream_check_device_status(void *cuda_stream);
  */
 stream_status stream_selftest_bounded_wait(int64_t limit_cycles, void *workspace, size_t workspace_bytes,
                                            void *cuda_stream);
+
+/* What stream_probe_unit_rates measured. */
+typedef struct {
+    double tma_bytes_per_clk;   /* bytes per SM clock that one SM's TMA unit brought from L2 into its shared
+                                   memory (16 KiB bulk copies of L2-resident data, four in flight, every SM
+                                   busy at once; CTA 0's figure) */
+    double mma_cycles_m128n64;  /* SM clocks per tcgen05.mma of M = 128, N = 64, K = 16, bf16, shared-memory
+                                   operands, issued back to back (32 would be the tensor core's own time) */
+    uint32_t error;             /* 0, or the code of a bounded wait that ran out (911 copies, 912 MMAs) */
+    uint32_t reserved;
+} stream_unit_rates;
+
+/*
+ * Measurement aid (the paper has no counterpart): the two unit rates that bound the tensor-core
+ * mask and attention kernels on the device at hand, so that a measured throughput can be set
+ * against what the SM delivers rather than against a data-sheet figure. Launches two short
+ * kernels (one CTA per SM, a few hundred microseconds), waits for `cuda_stream` and fills
+ * *out_host. Every wait inside is bounded like the product kernels' (STREAM_ERR_DEVICE_CHECK and
+ * out_host->error if one ran out).
+ *
+ *   scratch       device, 256-byte aligned, >= stream_probe_scratch_bytes(); overwritten (zeros:
+ *                 the source of the copies and a result record)
+ *   out_host      host
+ */
+size_t stream_probe_scratch_bytes(void);
+stream_status stream_probe_unit_rates(void *scratch, size_t scratch_bytes, stream_unit_rates *out_host, void *cuda_stream);
 
 /*
  * Bytes of device staging stream_run_host and stream_run_host_var need: room for Q, K, V, the mask,

@@ -23,15 +23,16 @@ struct Geom {
     long long ks_b, ks_h, ks_t;
 };
 
-// Header at the start of the mask workspace. The first 32 bytes mirror stream_stats.
+// Header at the start of the mask workspace. The first 40 bytes mirror stream_stats.
 struct WorkspaceHeader {
     unsigned long long tiles_scored;
     unsigned long long rows;
     unsigned int error;
     unsigned int error_info;
     unsigned long long tile_products;  // 64 x 64 tile products computed (more than tiles_scored where rows share a product)
+    unsigned long long tiles_fetched;  // tiles copied into shared memory (the tensor-core block kernel counts them)
     unsigned int work_counter;  // next work item of the persistent kernels
-    unsigned int pad[55];
+    unsigned int pad[53];
 };
 static_assert(sizeof(WorkspaceHeader) == 256, "workspace header is 256 bytes");
 

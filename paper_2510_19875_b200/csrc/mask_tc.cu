@@ -117,10 +117,14 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
                               unsigned k_smem, int which) {
     Ring st;
     unsigned grp_par = 0, jr_par[kR] = {0, 0, 0, 0};
+    unsigned long long fetched = 0;  // tiles this warp has asked TMA for
     for (;;) {
         if (!mbar_wait_w(smem_u32(&tl->jobs_ready[kR]), grp_par, tl, P.ws, 101)) return;
         grp_par ^= 1;
-        if (tl->grp_id < 0) return;
+        if (tl->grp_id < 0) {
+            if (elect_one()) atomicAdd(&P.ws->tiles_fetched, fetched);
+            return;
+        }
         const int b = tl->grp_b, kvh = tl->grp_kvh, qb = tl->grp_qb, h0 = tl->grp_h0, R = tl->grp_R;
         const int levels = tl->grp_levels;
         // Q tiles of the group's rows (previous group's MMAs are all complete by now)
@@ -130,6 +134,7 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
                 for (int c = 0; c < 2; ++c)
                     tma_load_4d(q_smem + (c * kR + r) * kHalfTile, tq, smem_u32(&tl->q_full), c * 64, qb * kBlk, h0 + r, b);
         }
+        if (which == 0 && tl->grp_new_q) fetched += (unsigned)R;
         __syncwarp();
         for (int level = 0; level < levels; ++level) {
             const int lists = level == 0 ? 1 : R;
@@ -144,6 +149,7 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
                     if ((st.idx & (kProducers - 1)) != which) { st.advance(kStages); continue; }  // the other producer's buffer
                     if (!mbar_wait_w(smem_u32(&tl->empty[st.idx]), st.phase ^ 1, tl, P.ws, 103)) return;
                     const int two = (j + 1 < n);
+                    fetched += 1u + (unsigned)two;
                     const int blk0 = tl->jobs_blk[li][j], blk1 = two ? tl->jobs_blk[li][j + 1] : 0;
                     if (elect_one()) {
                         const unsigned bar = smem_u32(&tl->full[st.idx]);

@@ -40,7 +40,15 @@ class StreamStats(ctypes.Structure):
     """``stream_stats`` of stream.h."""
 
     _fields_ = [("tiles_scored", ctypes.c_uint64), ("rows", ctypes.c_uint64), ("error", ctypes.c_uint32),
-                ("error_info", ctypes.c_uint32), ("tile_products", ctypes.c_uint64)]
+                ("error_info", ctypes.c_uint32), ("tile_products", ctypes.c_uint64),
+                ("tiles_fetched", ctypes.c_uint64)]
+
+
+class StreamUnitRates(ctypes.Structure):
+    """``stream_unit_rates`` of stream.h."""
+
+    _fields_ = [("tma_bytes_per_clk", ctypes.c_double), ("mma_cycles_m128n64", ctypes.c_double),
+                ("error", ctypes.c_uint32), ("reserved", ctypes.c_uint32)]
 
 
 class StreamError(RuntimeError):
@@ -86,6 +94,10 @@ def _load():
     lib.stream_effective_k.argtypes = [ctypes.c_int64, ctypes.c_int32, ctypes.c_double, ctypes.POINTER(ctypes.c_int32)]
     lib.stream_selftest_bounded_wait.restype = ctypes.c_int
     lib.stream_selftest_bounded_wait.argtypes = [ctypes.c_int64, vp, sz, vp]
+    lib.stream_probe_scratch_bytes.restype = sz
+    lib.stream_probe_scratch_bytes.argtypes = []
+    lib.stream_probe_unit_rates.restype = ctypes.c_int
+    lib.stream_probe_unit_rates.argtypes = [vp, sz, ctypes.POINTER(StreamUnitRates), vp]
     lib.stream_build_mask_static.restype = ctypes.c_int
     lib.stream_build_mask_static.argtypes = [P, vp, vp, vp, vp, vp]
     lib.stream_sparse_attention.restype = ctypes.c_int
@@ -182,6 +194,16 @@ def stream_effective_k(T: int, block_q: int, s: float) -> int:
 def stream_selftest_bounded_wait(limit_cycles: int, workspace, workspace_bytes: int, stream=None) -> None:
     """Diagnostic kernel whose bounded wait runs out after ``limit_cycles``; read the outcome with stream_read_stats."""
     _raise(_load().stream_selftest_bounded_wait(int(limit_cycles), _addr(workspace), workspace_bytes, _stream_handle(stream)))
+
+
+def stream_probe_scratch_bytes() -> int:
+    return int(_load().stream_probe_scratch_bytes())
+
+
+def stream_probe_unit_rates(scratch, scratch_bytes: int, stream=None) -> StreamUnitRates:
+    out = StreamUnitRates()
+    _raise(_load().stream_probe_unit_rates(_addr(scratch), scratch_bytes, ctypes.byref(out), _stream_handle(stream)))
+    return out
 
 
 def stream_build_mask_static(p: StreamProblem, q, k, mask_out, score_out, stream=None) -> None:
@@ -405,3 +427,12 @@ def effective_k(T: int, block_q: int, s: float) -> int:
     """Sparsity constant for an effective sparsity ``s`` in [0, 1] (Section 4.2 of the paper), as
     computed by the library's ``stream_effective_k``."""
     return stream_effective_k(T, block_q, s)
+
+
+def probe_unit_rates(device="cuda", stream=None) -> StreamUnitRates:
+    """TMA gather rate and tensor-core instruction time of the current device (``stream_probe_unit_rates``)."""
+    n = stream_probe_scratch_bytes()
+    if n == 0:
+        raise RuntimeError("no CUDA device to probe")
+    scratch = torch.empty(n, dtype=torch.uint8, device=device)
+    return stream_probe_unit_rates(scratch, n, stream)

@@ -143,6 +143,16 @@ def test_selftest_wait_rejects_bad_arguments_on_the_host(S):
         assert e.value.status == S.STREAM_ERR_WORKSPACE
 
 
+def test_unit_rate_probe_rejects_bad_arguments_on_the_host(S):
+    lib = S._load()
+    # no result record: refused before the device is even looked at
+    assert lib.stream_probe_unit_rates(256, 1 << 30, None, None) == S.STREAM_ERR_INVALID_ARG
+    out = S.StreamUnitRates()
+    rc = lib.stream_probe_unit_rates(None, 0, ctypes.byref(out), None)
+    assert rc in (S.STREAM_ERR_WORKSPACE, S.STREAM_ERR_CUDA)   # CUDA where there is no device to ask for its SM count
+    assert S.stream_probe_scratch_bytes() % 256 == 0
+
+
 @pytest.mark.parametrize("kw,s", [
     (dict(T=5000, k_top=9), 0.1), (dict(T=4096, k_top=32, causal=0), 0.3), (dict(T=777, block_q=16, block_k=16, d=64, k_top=5), 0.05),
     (dict(T=1000, block_q=32, block_k=8, d=64, k_top=12), 0.2), (dict(T=64, k_top=3), 0.9),

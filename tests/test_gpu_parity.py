@@ -624,3 +624,22 @@ def test_a_bounded_wait_that_runs_out_is_reported(S):
     assert ws.cpu().numpy().view(np.uint32)[4] == 901
     w = wl.generate(tc_spec(T=2048, k_top=4))
     assert_mask_parity(S, w, None, impl="tensor", score_cache=False)
+
+
+@pytest.mark.gpu
+def test_unit_rate_probe_and_fetch_counter(S):
+    """The measurement aid returns the two unit rates in the range this architecture can have
+    (a tcgen05.mma of M = 128, N = 64, K = 16 needs at least its 32 tensor-core clocks; the TMA
+    unit of one SM brings some tens of bytes per clock from L2), leaves the context usable, and the
+    tensor-core block kernel's fetch counter lies between a quarter of the tiles scored (every
+    fetched tile shared by the four heads of a kv head) and all of them."""
+    r = S.probe_unit_rates()
+    assert r.error == 0
+    assert 32.0 <= r.mma_cycles_m128n64 <= 80.0, r.mma_cycles_m128n64
+    assert 16.0 <= r.tma_bytes_per_clk <= 128.0, r.tma_bytes_per_clk
+    w = wl.generate(tc_spec(T=4096, k_top=8, n_q_heads=8, n_kv_heads=2))
+    q, k, _ = w.torch_tensors("cuda")
+    res = S.build_mask(q, k, block_q=64, block_k=64, k_top=8, impl="tensor")
+    st = res.stats()
+    q_tiles = 8 * 64   # one query tile per row
+    assert st.tiles_scored // 4 + q_tiles <= st.tiles_fetched <= st.tiles_scored + q_tiles, (st.tiles_fetched, st.tiles_scored)

@@ -72,6 +72,7 @@ struct Tail {
     unsigned long long x_bar[4];  // the two softmax warps of a lane quarter (one per group) meet here
     unsigned int tmem_base;
     int abort_flag;
+    int m_count[kMaskSlots];  // kept entries of the pair in each mask slot
 };
 // Dynamic shared memory: Q | P of group 0, P of group 1 | V stages | K stages | Tail | mask rows
 // [kMaskSlots][2][row_stride] (-1 where a row has nothing), the operands 1024-byte aligned.
@@ -133,25 +134,13 @@ __device__ __forceinline__ Item decode_item(const Params &P, int id) {
 // Entry e of the two rows: key block per row (negative = this row has nothing at e). An entry
 // is processed if either row has a block there. `rows` is the pair's shared copy [2][stride].
 struct Entry { int a, b; };
-__device__ __forceinline__ int next_entry(const int *rows, int stride, int e, int k_top, Entry *x) {
-    for (++e; e < k_top; ++e) {
-        x->a = rows[e];
-        x->b = rows[stride + e];
-        if (x->a >= 0 || x->b >= 0) return e;
-    }
-    return k_top;
-}
-
-// Number of kept entries of a pair, counted by a converged warp (32 entries per ballot).
-__device__ __forceinline__ int count_entries(const int *rows, int stride, int k_top) {
-    const int lane = threadIdx.x & 31;
-    int n = 0;
-    for (int base = 0; base < k_top; base += 32) {
-        const int e = base + lane;
-        const bool kept = e < k_top && (rows[e] >= 0 || rows[stride + e] >= 0);
-        n += __popc(__ballot_sync(0xffffffffu, kept));
-    }
-    return n;
+// The mask loader keeps only the kept entries of a pair, in order, at the front of the two
+// resident rows and leaves their number in the Tail: entry n of a pair is (rows[n], rows[stride + n]).
+__device__ __forceinline__ Entry entry_at(const int *rows, int stride, int n) {
+    Entry x;
+    x.a = rows[n];
+    x.b = rows[stride + n];
+    return x;
 }
 
 // ----------------------------------------------------------------------------------------------
@@ -167,12 +156,30 @@ __device__ void mask_loader_role(const Params &P, Tail *tl, int lane) {
         const int32_t *m0 = P.mask + (((long long)it.b * g.H + it.h0) * g.n_qb + it.qb) * g.k_top;
         const int32_t *m1 = m0 + (long long)g.n_qb * g.k_top;
         int *dst = mask_rows(tl, P, ms.idx);
-        for (int e = lane; e < g.k_top; e += 32) {
-            dst[e] = __ldg(m0 + e);
-            dst[P.row_stride + e] = it.R == 2 ? __ldg(m1 + e) : -1;
+        // an entry is kept if either row has a block there; the kept ones move to the front, so that
+        // the other roles index them instead of searching (their serial code is the kernel's pace)
+        int cnt = 0;
+        for (int base = 0; base < g.k_top; base += 32) {
+            const int e = base + lane;
+            int a = -1, b = -1;
+            if (e < g.k_top) {
+                a = __ldg(m0 + e);
+                if (it.R == 2) b = __ldg(m1 + e);
+            }
+            const bool kept = a >= 0 || b >= 0;
+            const unsigned bal = __ballot_sync(0xffffffffu, kept);
+            if (kept) {
+                const int pos = cnt + __popc(bal & ((1u << lane) - 1u));
+                dst[pos] = a;
+                dst[P.row_stride + pos] = b;
+            }
+            cnt += __popc(bal);
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&tl->m_full[ms.idx]));
+        if (lane == 0) {
+            tl->m_count[ms.idx] = cnt;
+            mbar_arrive(smem_u32(&tl->m_full[ms.idx]));
+        }
         ms.advance(kMaskSlots);
     }
 }
@@ -183,7 +190,8 @@ __device__ void mask_loader_role(const Params &P, Tail *tl, int lane) {
 // converged (lane 0's probe result is broadcast) and one elected lane issues.
 struct LoadStream {
     int id;            // pair being walked
-    int e;             // current entry (k_top = pair exhausted), -2 = pair not opened yet
+    int e;             // current entry (n = pair exhausted), -2 = pair not opened yet
+    int n;             // kept entries of the pair
     int n_issued;      // loads issued for this pair
     Entry cur;
     Item it;
@@ -197,7 +205,6 @@ __device__ __forceinline__ bool probe_w(unsigned bar, unsigned parity) {
 
 __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUtensorMap *tk, const CUtensorMap *tv,
                               Tail *tl, unsigned q_smem, unsigned k_smem, unsigned v_smem) {
-    const Geom &g = P.g;
     unsigned q_par = 0;
     LoadStream K, V;
     K.id = V.id = blockIdx.x;
@@ -226,12 +233,14 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
         if (S.e == -2) {  // open the pair: its mask rows must be resident
             if (!probe_w(smem_u32(&tl->m_full[S.ms.idx]), S.ms.phase)) return false;
             S.it = decode_item(P, S.id);
-            S.e = next_entry(rows, P.row_stride, -1, g.k_top, &S.cur);
-            S.q_due = is_k && S.e < g.k_top;  // (a pair with nothing kept: only the softmax warps act)
+            S.n = tl->m_count[S.ms.idx];
+            S.e = 0;
+            if (S.n > 0) S.cur = entry_at(rows, P.row_stride, 0);
+            S.q_due = is_k && S.n > 0;  // (a pair with nothing kept: only the softmax warps act)
             S.n_issued = 0;
             return true;
         }
-        if (S.e >= g.k_top && !S.q_due) {  // pair exhausted: give its mask rows back, go to the next one
+        if (S.e >= S.n && !S.q_due) {  // pair exhausted: give its mask rows back, go to the next one
             if (elect_one()) mbar_arrive(smem_u32(&tl->m_empty[S.ms.idx]));
             __syncwarp();
             S.ms.advance(kMaskSlots);
@@ -240,13 +249,13 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
             return true;
         }
         if (is_k) {
-            if (S.e < g.k_top && !(S.q_due && S.n_issued > 0)) {
+            if (S.e < S.n && !(S.q_due && S.n_issued > 0)) {
                 // a K stage is free once the logits computed from it are complete
                 if (!probe_w(smem_u32(&tl->k_empty[S.ring.idx]), S.ring.phase ^ 1)) return false;
                 if (elect_one()) load_k_pair(k_smem + S.ring.idx * kOperand, smem_u32(&tl->k_full[S.ring.idx]), S.it, S.cur);
                 __syncwarp();
                 S.ring.advance(P.n_k_stages);
-                S.e = next_entry(rows, P.row_stride, S.e, g.k_top, &S.cur);
+                if (++S.e < S.n) S.cur = entry_at(rows, P.row_stride, S.e);
                 ++S.n_issued;
                 return true;
             }
@@ -267,7 +276,7 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
         if (elect_one()) load_v_pair(v_smem + S.ring.idx * kOperand, smem_u32(&tl->v_full[S.ring.idx]), S.it, S.cur);
         __syncwarp();
         S.ring.advance(P.n_v_stages);
-        S.e = next_entry(rows, P.row_stride, S.e, g.k_top, &S.cur);
+        if (++S.e < S.n) S.cur = entry_at(rows, P.row_stride, S.e);
         return true;
     };
     long long t_last = clock64();
@@ -297,15 +306,13 @@ __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUte
 
 // S_g = [Q_0; Q_1] [K_a; K_b]^T for every kept entry (g = the entry's number within its pair % 2).
 __device__ void qk_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_smem, unsigned tmem_base) {
-    const Geom &g = P.g;
     Ring ks, ms;
     unsigned cnt[2] = {0, 0};  // entries each group has had over the whole kernel
     unsigned q_par = 0;
     const unsigned q_lo = desc_lo_sw128(q_smem, 16), k_lo = desc_lo_sw128(k_smem, 16);
     for (int id = blockIdx.x; id < P.n_items; id += gridDim.x) {
         if (!wait_w(smem_u32(&tl->m_full[ms.idx]), ms.phase, tl, 207)) return;
-        const int *rows = mask_rows(tl, P, ms.idx);
-        const int n_entries = count_entries(rows, P.row_stride, g.k_top);  // the issuers need no more than the count
+        const int n_entries = tl->m_count[ms.idx];  // the issuers need no more than the count
         if (n_entries > 0) {
             if (!wait_w(smem_u32(&tl->q_full), q_par, tl, 201)) return;
             q_par ^= 1;
@@ -339,15 +346,13 @@ __device__ void qk_role(const Params &P, Tail *tl, unsigned q_smem, unsigned k_s
 
 // O_g (+)= P_g [V_a; V_b] for every kept entry; a group's first entry of a pair starts its O afresh.
 __device__ void pv_role(const Params &P, Tail *tl, unsigned p_smem, unsigned v_smem, unsigned tmem_base) {
-    const Geom &g = P.g;
     Ring vs, ms;  // vs: the entry's V stage
     unsigned cnt[2] = {0, 0};  // entries each group has had over the whole kernel
     // the MN-major V tiles have their two 64-channel halves kHalfTile apart
     const unsigned p_lo = desc_lo_sw128(p_smem, 16), v_lo = desc_lo_sw128(v_smem, kHalfTile);
     for (int id = blockIdx.x; id < P.n_items; id += gridDim.x) {
         if (!wait_w(smem_u32(&tl->m_full[ms.idx]), ms.phase, tl, 208)) return;
-        const int *rows = mask_rows(tl, P, ms.idx);
-        const int n_entries = count_entries(rows, P.row_stride, g.k_top);
+        const int n_entries = tl->m_count[ms.idx];
         unsigned fresh = 3u;  // bit g: group g has not added anything for this pair yet
         for (int i = 0; i < n_entries; ++i) {
             if (!wait_w(smem_u32(&tl->v_full[vs.idx]), vs.phase, tl, 205)) return;
@@ -429,11 +434,9 @@ __device__ void softmax_role(const Params &P, Tail *tl, unsigned char *p_ptr, un
         const int *rows = mask_rows(tl, P, ms.idx);
         float ref = -CUDART_INF_F, l = 0.f;
         bool pending = false;  // a P V chain of this group and pair may still be running
-        Entry cur;
-        unsigned n = 0;
-        for (int e = next_entry(rows, P.row_stride, -1, g.k_top, &cur); e < g.k_top;
-             e = next_entry(rows, P.row_stride, e, g.k_top, &cur), ++n) {
-            if ((int)(n & 1u) != grp) continue;  // n: the entry's number within the pair
+        const int n_entries = tl->m_count[ms.idx];
+        const int *my_row = rows + half * P.row_stride;  // this token's row of the pair
+        for (int n = grp; n < n_entries; n += 2) {  // entry n of a pair belongs to group n % 2
             // the token's 64 logits against its row's key block
             if (!wait_w(s_full, s_par, tl, 301)) return;
             s_par ^= 1;
@@ -446,7 +449,7 @@ __device__ void softmax_role(const Params &P, Tail *tl, unsigned char *p_ptr, un
             __syncwarp();
             if (lane == 0) mbar_arrive(s_empty);
             // keys of the block this token may attend: a prefix of n_hi keys (inside T, not after it if causal)
-            const int blk = half ? cur.b : cur.a;
+            const int blk = my_row[n];
             int n_hi = 0;
             if (blk >= 0 && row_active) {
                 const long long k0 = (long long)blk * kBlk;

@@ -433,6 +433,7 @@ __device__ void softmax_role(const Params &P, Tail *tl, unsigned char *p_ptr, un
         if (!wait_w(smem_u32(&tl->m_full[ms.idx]), ms.phase, tl, 305)) return;
         const int *rows = mask_rows(tl, P, ms.idx);
         float ref = -CUDART_INF_F, l = 0.f;
+        bool ref_open = true;  // some token of this warp has no reference yet (the same in every lane)
         bool pending = false;  // a P V chain of this group and pair may still be running
         const int n_entries = tl->m_count[ms.idx];
         const int *my_row = rows + half * P.row_stride;  // this token's row of the pair
@@ -496,9 +497,10 @@ __device__ void softmax_role(const Params &P, Tail *tl, unsigned char *p_ptr, un
                 return max_of_64(x);
             };
             // the token's first allowed logits set its reference (once per pair)
-            if (__any_sync(0xffffffffu, ref == -CUDART_INF_F && n_hi > 0)) {
+            if (ref_open && __any_sync(0xffffffffu, ref == -CUDART_INF_F && n_hi > 0)) {
                 const float mx = masked_max();
                 if (ref == -CUDART_INF_F) ref = mx;
+                ref_open = __any_sync(0xffffffffu, ref == -CUDART_INF_F);
             }
             make_p(ref == -CUDART_INF_F ? 0.f : -ref * P.scale_log2);
             const bool redo = !(esum <= kLazySum);

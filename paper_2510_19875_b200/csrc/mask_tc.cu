@@ -15,9 +15,9 @@
 // only right branches are fetched. With several k per call a group runs the hierarchy once per
 // k on the same Q tiles and fetches only blocks whose score it does not have yet.
 //
-// Roles (512 threads, the last two warps idle): warp 0 TMA producer, warps 1, 3, 12, 13 MMA
-// issuers (warp 1 owns TMEM), warp 2 controller, warps 4..7 and 8..11 the two epilogue groups
-// (TMEM lane quarter = warp % 4). All roles walk the same fixed unit order (level 1: stage-major,
+// Roles (512 threads, the last warp idle): warps 0 and 14 TMA producers (even and odd stage
+// buffers; warp 0 also brings the Q tiles), warps 1, 3, 12, 13 MMA issuers (warp 1 owns TMEM),
+// warp 2 controller, warps 4..7 and 8..11 the two epilogue groups (TMEM lane quarter = warp % 4). All roles walk the same fixed unit order (level 1: stage-major,
 // row-minor; later levels: row-major), synchronised by mbarriers only. Every wait is bounded: on
 // a timeout the CTA records an error code in the workspace header, raises a shared abort flag,
 // drains its own copies and leaves.
@@ -111,8 +111,10 @@ __device__ __forceinline__ unsigned long long cache_pack(unsigned tag, float s) 
 // ----------------------------------------------------------------------------------------------
 // Roles
 // ----------------------------------------------------------------------------------------------
-// Run by all 32 lanes of warp 0, converged (warp-wide waits, one elected lane issues): a single
-// diverged lane issues TMA copies several times more slowly.
+// Run by all 32 lanes of a producer warp, converged (warp-wide waits, one elected lane issues): a
+// single diverged lane issues TMA copies several times more slowly. Two producers share the
+// stages by buffer parity: one alone is busy more than half of the time with the four copies and
+// the barrier arm of a stage, and the issuing warps then wait for data.
 __device__ void producer_role(const Params &P, const CUtensorMap *tq, const CUtensorMap *tk, Tail *tl, unsigned q_smem,
                               unsigned k_smem, int which) {
     Ring st;

@@ -244,23 +244,50 @@ __host__ __device__ constexpr unsigned idesc_bf16(unsigned M, unsigned N, bool b
 
 // Top-k of the (up to) 64 candidates a warp holds two per lane (a node's left and right branch):
 // keep the k best by (score descending, candidate index ascending), the candidates numbered
-// 2 * lane (left) and 2 * lane + 1 (right). Rank by counting, with shuffles.
+// 2 * lane (left) and 2 * lane + 1 (right); k <= 32.
+//
+// The k-th largest score is found with a sorting network instead of counting ranks (4096
+// comparisons, which made this the longest step of a row's level): the scores become unsigned
+// keys of the same order (-0 first brought to +0, so that equal floats give equal keys; an absent
+// candidate gets key 0, below every score), the 32 left keys are sorted descending and the 32
+// right keys ascending across the lanes (one bitonic network, 15 exchange steps, both registers
+// at once), the lane-wise maximum of the two is then the 32 largest keys as a bitonic sequence,
+// five more steps sort it, and lane k - 1 holds the threshold. Every candidate above the threshold
+// is kept; of those equal to it the first ones in candidate order, as many as are still missing.
 struct Keep { bool l, r; };
+__device__ __forceinline__ unsigned score_key(bool valid, float s) {
+    const unsigned b = __float_as_uint(s + 0.f);
+    return valid ? (b ^ ((b & 0x80000000u) ? 0xffffffffu : 0x80000000u)) : 0u;
+}
 __device__ __forceinline__ Keep select_topk(bool vl, float sl, bool vr, float sr, int k, int lane) {
     const int total = __popc(__ballot_sync(0xffffffffu, vl)) + __popc(__ballot_sync(0xffffffffu, vr));
     if (total <= k) return {vl, vr};
-    const float ninf = __int_as_float(0xff800000);
-    const float el = vl ? sl : ninf, er = vr ? sr : ninf;
-    int rank_l = 0, rank_r = 0;
-#pragma unroll 8
-    for (int j = 0; j < 32; ++j) {
-        const float ol = __shfl_sync(0xffffffffu, el, j), orr = __shfl_sync(0xffffffffu, er, j);
-        rank_l += (ol > el) || (ol == el && j < lane);
-        rank_l += (orr > el) || (orr == el && j < lane);
-        rank_r += (ol > er) || (ol == er && j <= lane);
-        rank_r += (orr > er) || (orr == er && j < lane);
+    const unsigned kl = score_key(vl, sl), kr = score_key(vr, sr);
+    unsigned a = kl, b = kr;  // a: sorted descending over the lanes, b: ascending
+#pragma unroll
+    for (int k2 = 2; k2 <= 32; k2 <<= 1) {
+#pragma unroll
+        for (int j = k2 >> 1; j > 0; j >>= 1) {
+            const unsigned oa = __shfl_xor_sync(0xffffffffu, a, j), ob = __shfl_xor_sync(0xffffffffu, b, j);
+            // in an ascending network the lower lane of a pair takes the minimum inside an "up" block
+            const bool first = (((lane & j) == 0) == ((lane & k2) == 0));
+            a = first ? max(a, oa) : min(a, oa);
+            b = first ? min(b, ob) : max(b, ob);
+        }
     }
-    return {vl && rank_l < k, vr && rank_r < k};
+    unsigned c = max(a, b);  // the 32 largest of the 64 keys, a bitonic sequence over the lanes
+#pragma unroll
+    for (int j = 16; j > 0; j >>= 1) {
+        const unsigned oc = __shfl_xor_sync(0xffffffffu, c, j);
+        c = ((lane & j) == 0) ? max(c, oc) : min(c, oc);
+    }
+    const unsigned thr = __shfl_sync(0xffffffffu, c, k - 1);  // the k-th largest key (with multiplicity)
+    const bool gl = kl > thr, gr = kr > thr, el = kl == thr, er = kr == thr;
+    const int missing = k - __popc(__ballot_sync(0xffffffffu, gl)) - __popc(__ballot_sync(0xffffffffu, gr));
+    const unsigned bel = __ballot_sync(0xffffffffu, el), ber = __ballot_sync(0xffffffffu, er);
+    const unsigned lt = (1u << lane) - 1u;
+    const int pos_l = __popc(bel & lt) + __popc(ber & lt), pos_r = pos_l + (el ? 1 : 0);
+    return {vl && (gl || (el && pos_l < missing)), vr && (gr || (er && pos_r < missing))};
 }
 
 struct Ring {  // position in a ring of barriers with phase tracking

@@ -5,7 +5,7 @@ import numpy as np
 import pytest
 import torch
 
-from helpers import check_mask_invariants, compare_masks, oracle_problem, sample_rows
+from helpers import TIE_GAP, check_mask_invariants, compare_masks, oracle_problem, sample_rows
 from oracle import stream_oracle as so
 from paper_2510_19875_b200 import workloads as wl
 
@@ -643,3 +643,49 @@ def test_unit_rate_probe_and_fetch_counter(S):
     st = res.stats()
     q_tiles = 8 * 64   # one query tile per row
     assert st.tiles_scored // 4 + q_tiles <= st.tiles_fetched <= st.tiles_scored + q_tiles, (st.tiles_fetched, st.tiles_scored)
+
+
+def integer_workload(spec, lo=-2, hi=2):
+    """Q and K with small integer entries (exact in bf16 and fp32): every dot product is an integer
+    that fp32 accumulation and the oracle's fp64-then-round give alike, so tile maxima coincide
+    exactly on both sides and many branches tie."""
+    w = wl.generate(spec, with_v=False)
+    rng = np.random.default_rng(spec.seed + 1000)
+    def ints(shape):
+        x = rng.integers(lo, hi + 1, size=shape).astype(np.float32)
+        return wl.to_bf16_bits(x) if spec.dtype == "bf16" else x
+    w.q = ints(w.q.shape)
+    w.k = ints(w.k.shape)
+    return w
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("kw,impl,bq", [
+    (dict(T=4096, k_top=8, n_q_heads=4, n_kv_heads=1), "tensor", 64),     # tcgen05 block kernel, 3 levels
+    (dict(T=8192, k_top=32, n_q_heads=8, n_kv_heads=2), "tensor", 64),    # k = 32: all 64 candidates of a level compete
+    (dict(T=5000, k_top=5, n_q_heads=3, n_kv_heads=1), "tensor", 64),     # ragged T, odd k
+    (dict(T=4096, k_top=8, n_q_heads=4, n_kv_heads=1), "generic", 64),    # fp32-FMA kernel on the same inputs
+    (dict(T=2048, k_top=16, n_q_heads=2, n_kv_heads=1), "auto", 1),       # per-token tensor-core kernel
+])
+def test_exact_ties_are_broken_by_block_index(S, kw, impl, bq):
+    """With integer inputs the scores are exact on both sides and ties between branches are the
+    rule, so nothing is exempt: every row must be the oracle's row, which keeps, among equal
+    scores, the lower block index - and the scores of the kept blocks must be equal bit for bit."""
+    spec = tc_spec(**kw)
+    w = integer_workload(spec)
+    res = run_mask(S, w, impl=impl, block_q=bq, want_scores=True)
+    st = res.stats()
+    assert st.error == 0
+    mask = res.mask.cpu().numpy()
+    flat = mask.reshape(-1, mask.shape[-1])
+    p = oracle_problem(spec, block_q=bq)
+    n_rows = flat.shape[0]
+    rows = None if n_rows <= 4096 else np.unique(np.concatenate([np.arange(64), np.arange(n_rows - 64, n_rows),
+                                                                  np.random.default_rng(3).choice(n_rows, 2048, replace=False)]))
+    ora = so.build_mask_rows(p, w.q, w.k, rows, want_scores=True)
+    got = flat if rows is None else flat[rows]
+    assert (ora["min_gap"] < TIE_GAP).mean() > 0.1          # the case is what it says: exact ties at the cut are common
+    np.testing.assert_array_equal(got, ora["mask"])
+    sc = res.scores.cpu().numpy().reshape(-1, mask.shape[-1])
+    sc = sc if rows is None else sc[rows]
+    np.testing.assert_array_equal(sc, ora["scores"])

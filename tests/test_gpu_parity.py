@@ -689,3 +689,28 @@ def test_exact_ties_are_broken_by_block_index(S, kw, impl, bq):
     sc = res.scores.cpu().numpy().reshape(-1, mask.shape[-1])
     sc = sc if rows is None else sc[rows]
     np.testing.assert_array_equal(sc, ora["scores"])
+
+
+@pytest.mark.gpu
+def test_exact_ties_in_the_several_k_and_variable_k_builds(S):
+    """The same integer inputs through the several-k build (scores taken from the score memory in
+    the later passes) and the variable-k build: every row, every k, bit for bit."""
+    spec = tc_spec(T=4096, k_top=16, n_q_heads=8, n_kv_heads=2)
+    w = integer_workload(spec)
+    q, k, _ = w.torch_tensors("cuda")
+    p = oracle_problem(spec)
+    k_list = [16, 8, 3]
+    res = S.build_masks(q, k, k_list, block_q=64, block_k=64, impl="tensor", want_scores=True)
+    torch.cuda.synchronize()
+    assert res.stats().error == 0
+    ora = so.build_mask_rows_multi(p, w.q, w.k, k_list, want_scores=True)
+    np.testing.assert_array_equal(res.mask.cpu().numpy().reshape(len(k_list), -1, p.k_top), ora["mask"])
+    np.testing.assert_array_equal(res.scores.cpu().numpy().reshape(len(k_list), -1, p.k_top), ora["scores"])
+    nqb = so.num_query_blocks(p)
+    k_row = (1 + (np.arange(nqb) * 5) % 16).astype(np.int32)
+    var = S.build_mask(q, k, block_q=64, block_k=64, k_top=16, k_row=torch.from_numpy(k_row).cuda(), impl="tensor", want_scores=True)
+    torch.cuda.synchronize()
+    assert var.stats().error == 0
+    orv = so.build_mask_rows_var(p, w.q, w.k, k_row, want_scores=True)
+    np.testing.assert_array_equal(var.mask.cpu().numpy().reshape(-1, p.k_top), orv["mask"])
+    np.testing.assert_array_equal(var.scores.cpu().numpy().reshape(-1, p.k_top), orv["scores"])

@@ -181,9 +181,9 @@ def ncu_traffic(kernel: str, spec):
 
 
 # The two SM units the tensor-core kernels lean on, measured on the device by the library's own
-# probe (stream_probe_unit_rates) right before the timed steps: the bytes per clock one SM's TMA
-# unit brings from L2 into shared memory, and the clocks one tcgen05.mma of the mask kernel's
-# shape takes. The bench line sets each kernel's traffic and instruction count against them.
+# probe (stream_probe_unit_rates) right before the timed steps: the bytes per clock two issuing
+# warps bring from L2 into one SM's shared memory through TMA, and the clocks one tcgen05.mma of
+# the mask kernel's shape takes. The bench line sets each kernel's traffic and instruction count against them.
 TC_KERNELS = ("mask_tc_kernel", "attn_tc_kernel")
 
 

@@ -304,8 +304,8 @@ stream_status stream_selftest_bounded_wait(int64_t limit_cycles, void *workspace
 /* What stream_probe_unit_rates measured. */
 typedef struct {
     double tma_bytes_per_clk;   /* bytes per SM clock that one SM's TMA unit brought from L2 into its shared
-                                   memory (16 KiB bulk copies of L2-resident data, four in flight, every SM
-                                   busy at once; CTA 0's figure) */
+                                   memory (16 KiB bulk copies of L2-resident data, two issuing warps with
+                                   four copies in flight each, every SM busy at once; CTA 0's figure) */
     double mma_cycles_m128n64;  /* SM clocks per tcgen05.mma of M = 128, N = 64, K = 16, bf16, shared-memory
                                    operands, issued back to back (32 would be the tensor core's own time) */
     uint32_t error;             /* 0, or the code of a bounded wait that ran out (911 copies, 912 MMAs) */
